@@ -1,0 +1,245 @@
+"""fp64 CPU oracle for the AdapShot KV-reuse hot path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain statement of what the
+path computes, written from the paper's definitions.  Only the test-suite, the
+smoke check and the CPU-baseline / reference legs of the benchmark may import
+it.  It shares no code with the CUDA library and never imports the package.
+
+Every function works on numpy float64 arrays that hold the *stored* values of
+the inputs (fp32 or bf16 values widen to fp64 exactly) and accumulates in fp64.
+A matmul / sort from numpy may serve as one step; nothing is blocked, fused or
+reordered beyond what the cited definition states.
+
+Pins (tests/test_oracle_pins.py) tie each function to something other than
+itself: closed forms, the complex-number form of the rotation, brute-force
+loops, scipy routines, the paper's two-shot position example, and the
+relative-position invariance of rotary attention.
+
+Parity status: every function here is pinned.  (The two-token entropy variant
+of Eq. 2 and the attention-based relevance score of Eq. 5 are not implemented
+here; they are outside the hot path.)
+
+Notation (paper, Sec. 3-4): N shots of lengths T_i, k selected shots, Hq/Hkv
+heads, G = Hq/Hkv, d head_dim, T_q query tokens, L_j context length of probe j.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# Step 1: semantic relevance ranking (Sec. 4.1 "semantic relevance ranking",
+# Sec. 4.2 last paragraph "rank ... in descending order and select the top k";
+# the score itself is the cosine of embeddings, as the build's problem
+# statement fixes it).
+# --------------------------------------------------------------------------
+def cosine_scores(q_emb: np.ndarray, emb: np.ndarray) -> np.ndarray:
+    """s[b, i] = <q_b, e_i> / (|q_b| |e_i|); 0 where either norm is 0."""
+    q = np.asarray(q_emb, dtype=F64)
+    e = np.asarray(emb, dtype=F64)
+    dots = q @ e.T
+    qn = np.sqrt(np.sum(q * q, axis=1))
+    en = np.sqrt(np.sum(e * e, axis=1))
+    denom = qn[:, None] * en[None, :]
+    out = np.zeros_like(dots)
+    nz = denom > 0.0
+    out[nz] = dots[nz] / denom[nz]
+    return out
+
+
+def select_topk(q_emb: np.ndarray, emb: np.ndarray, k: int):
+    """Indices of the k most relevant shots per query, most relevant first.
+
+    Equal scores are ordered by the lower shot id (a stable sort on the
+    negated score).  Returns (sel_idx int32 [B, k], sel_score fp64 [B, k]).
+    """
+    s = cosine_scores(q_emb, emb)
+    B, N = s.shape
+    if not (1 <= k <= N):
+        raise ValueError("k must be in 1..N")
+    sel = np.empty((B, k), dtype=np.int32)
+    sc = np.empty((B, k), dtype=F64)
+    for b in range(B):
+        order = np.argsort(-s[b], kind="stable")[:k]
+        sel[b] = order
+        sc[b] = s[b, order]
+    return sel, sc
+
+
+def min_adjacent_gap(q_emb: np.ndarray, emb: np.ndarray, k: int) -> float:
+    """Smallest gap between neighbouring sorted scores among ranks 1..k+1.
+
+    A gap of exactly 0 is a true tie (decided by shot id) and is ignored; a
+    tiny non-zero gap marks a seed on which fp64 rounding order could decide.
+    """
+    s = cosine_scores(q_emb, emb)
+    best = np.inf
+    for b in range(s.shape[0]):
+        top = -np.sort(-s[b])[: k + 1]
+        gaps = top[:-1] - top[1:]
+        gaps = gaps[gaps > 0.0]
+        if gaps.size:
+            best = min(best, float(gaps.min()))
+    return best
+
+
+# --------------------------------------------------------------------------
+# Step 2: destination offsets (Sec. 4.3, two-shot example: shot B placed after
+# shot A occupies positions T_A .. T_A+T_B-1, its offset is Delta = T_A).
+# --------------------------------------------------------------------------
+def plan_offsets(sel_idx: np.ndarray, shot_off: np.ndarray) -> np.ndarray:
+    """ctx_off[b, r] = sum of the lengths of the first r selected shots."""
+    sel = np.asarray(sel_idx)
+    so = np.asarray(shot_off, dtype=np.int64)
+    B, k = sel.shape
+    ctx_off = np.zeros((B, k + 1), dtype=np.int64)
+    for b in range(B):
+        for r in range(k):
+            s = int(sel[b, r])
+            ctx_off[b, r + 1] = ctx_off[b, r] + (so[s + 1] - so[s])
+    return ctx_off
+
+
+# --------------------------------------------------------------------------
+# Step 3: rotary encoding and re-encoding (Sec. 4.3, Eq. 6 and Eq. 7).
+# --------------------------------------------------------------------------
+def rope_theta(d: int, base: float) -> np.ndarray:
+    """theta_i = base^(-2i/d), i = 0 .. d/2-1 (text after Eq. 6)."""
+    i = np.arange(d // 2, dtype=F64)
+    return np.power(F64(base), -2.0 * i / F64(d))
+
+
+def rotate_half(x: np.ndarray) -> np.ndarray:
+    """Half-split convention of the evaluated model families:
+    rotate_half(x) = [-x_{d/2..d-1}, x_{0..d/2-1}]."""
+    h = x.shape[-1] // 2
+    return np.concatenate([-x[..., h:], x[..., :h]], axis=-1)
+
+
+def rope(x: np.ndarray, p, base: float) -> np.ndarray:
+    """Eq. 6: RoPE(x, p) = x * cos(p theta) + rotate_half(x) * sin(p theta).
+
+    x [..., d]; p broadcastable to x.shape[:-1].  The d/2 angles are repeated
+    over both halves of the vector.  Eq. 7 is the same map with p = Delta.
+    """
+    x = np.asarray(x, dtype=F64)
+    d = x.shape[-1]
+    th = rope_theta(d, base)
+    ang = np.asarray(p, dtype=F64)[..., None] * th
+    c = np.concatenate([np.cos(ang), np.cos(ang)], axis=-1)
+    s = np.concatenate([np.sin(ang), np.sin(ang)], axis=-1)
+    return x * c + rotate_half(x) * s
+
+
+def assemble_kv(k_pool, v_pool, shot_off, sel_row, base: float, k_pos_mode: int = 0):
+    """Concatenate the selected shots' cached K/V in selection order and move K
+    to its new contiguous positions (Sec. 4.3; Eq. 7).
+
+    k_pool, v_pool : [n_layers, pool_tokens, Hkv, d]
+    sel_row        : [k] shot ids of ONE query, most relevant first
+    k_pos_mode 0   : pool K carries no position; the rotation angle of the
+                     token at new position o+t is (o+t) theta.
+    k_pos_mode 1   : pool K was rotated at its shot-local position t when the
+                     shot was prefilled alone from position 0, so the
+                     correction is Delta = o for the whole shot (Eq. 7).
+    V is copied unchanged.  Returns (k_ctx, v_ctx [n_layers, L, Hkv, d], ctx_off [k+1]).
+    """
+    k_pool = np.asarray(k_pool, dtype=F64)
+    v_pool = np.asarray(v_pool, dtype=F64)
+    so = np.asarray(shot_off, dtype=np.int64)
+    ctx_off = plan_offsets(np.asarray(sel_row)[None, :], so)[0]
+    n_layers, _, hkv, d = k_pool.shape
+    L = int(ctx_off[-1])
+    k_ctx = np.zeros((n_layers, L, hkv, d), dtype=F64)
+    v_ctx = np.zeros((n_layers, L, hkv, d), dtype=F64)
+    for r, s in enumerate(np.asarray(sel_row)):
+        a, b = int(so[s]), int(so[s + 1])
+        o = int(ctx_off[r])
+        T = b - a
+        t = np.arange(T, dtype=F64)
+        delta = (o + t) if k_pos_mode == 0 else np.full(T, F64(o))
+        # delta is per token; broadcast over layers and heads
+        k_ctx[:, o:o + T] = rope(k_pool[:, a:b], delta[None, :, None], base)
+        v_ctx[:, o:o + T] = v_pool[:, a:b]
+    return k_ctx, v_ctx, ctx_off
+
+
+# --------------------------------------------------------------------------
+# Step 4: probe attention (Eq. 1 context; tree mask of Sec. 4.1: probe j sees
+# its first n_j shots and, causally, its own tokens; scale 1/sqrt(d) of Eq. 5).
+# --------------------------------------------------------------------------
+def attn_row(q_row, kq, vq, k_ctx, v_ctx, L_j: int, t: int, kv_head: int,
+             base: float, scale: float | None = None):
+    """One output row: probe token t (position L_j + t), one query head.
+
+    q_row [d] un-rotated query vector of that head;  kq, vq [T_q, Hkv, d]
+    un-rotated keys / values of the probe's own tokens;  k_ctx, v_ctx
+    [L, Hkv, d] assembled cache of one layer (K already at positions 0..L-1).
+    Returns (out [d], lse) with lse = log sum exp of the scaled scores.
+    """
+    d = q_row.shape[-1]
+    sc = (1.0 / np.sqrt(F64(d))) if scale is None else F64(scale)
+    q = rope(np.asarray(q_row, dtype=F64), F64(L_j + t), base)
+    own_pos = L_j + np.arange(t + 1, dtype=F64)
+    k_own = rope(np.asarray(kq, dtype=F64)[: t + 1, kv_head], own_pos, base)
+    keys = np.concatenate([np.asarray(k_ctx, dtype=F64)[:L_j, kv_head], k_own], axis=0)
+    vals = np.concatenate([np.asarray(v_ctx, dtype=F64)[:L_j, kv_head],
+                           np.asarray(vq, dtype=F64)[: t + 1, kv_head]], axis=0)
+    s = (keys @ q) * sc
+    m = s.max()
+    e = np.exp(s - m)
+    z = e.sum()
+    return (e / z) @ vals, float(m + np.log(z))
+
+
+def query_attn(q, kq, vq, k_ctx, v_ctx, L_list, base: float, scale: float | None = None):
+    """All rows of all probes of one query at one layer.
+
+    q [P, T_q, Hq, d];  kq, vq [P, T_q, Hkv, d];  k_ctx, v_ctx [L, Hkv, d];
+    L_list[j] = context length of probe j.  Query head h reads KV head h // G.
+    Returns (out [P, T_q, Hq, d], lse [P, Hq, T_q]).
+    """
+    q = np.asarray(q, dtype=F64)
+    P, Tq, Hq, d = q.shape
+    Hkv = np.asarray(kq).shape[2]
+    G = Hq // Hkv
+    out = np.zeros((P, Tq, Hq, d), dtype=F64)
+    lse = np.zeros((P, Hq, Tq), dtype=F64)
+    for j in range(P):
+        for h in range(Hq):
+            for t in range(Tq):
+                o, l = attn_row(q[j, t, h], kq[j], vq[j], k_ctx, v_ctx,
+                                int(L_list[j]), t, h // G, base, scale)
+                out[j, t, h] = o
+                lse[j, h, t] = l
+    return out, lse
+
+
+# --------------------------------------------------------------------------
+# Step 5: confidence probe (Eq. 2, taken over the whole vocabulary; natural
+# log; the threshold rule of the paragraph after Eq. 2).
+# --------------------------------------------------------------------------
+def entropy(logits: np.ndarray) -> np.ndarray:
+    """H_r = -sum_v p_v ln p_v with p = softmax(logits_r); p = 0 terms add 0."""
+    x = np.asarray(logits, dtype=F64)
+    m = x.max(axis=-1, keepdims=True)
+    e = np.exp(x - m)
+    p = e / e.sum(axis=-1, keepdims=True)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        terms = np.where(p > 0.0, p * np.log(p), 0.0)
+    return -terms.sum(axis=-1)
+
+
+def first_ok(H: np.ndarray, tau: float, P: int) -> np.ndarray:
+    """Per group of P nested probes: index of the first probe with H <= tau,
+    -1 if none (the minimum shot count that satisfies the threshold)."""
+    Hm = np.asarray(H, dtype=F64).reshape(-1, P)
+    out = np.full(Hm.shape[0], -1, dtype=np.int32)
+    for b in range(Hm.shape[0]):
+        for j in range(P):
+            if Hm[b, j] <= tau:
+                out[b] = j
+                break
+    return out
