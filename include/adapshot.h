@@ -1,0 +1,169 @@
+/*
+ * adapshot.h - C ABI of the B200 (sm_100a) AdapShot KV-reuse hot path.
+ *
+ * The path (paper Sec. 4): rank the cached shots for a query and take the top k
+ * (Sec. 4.1/4.2), concatenate the selected shots' cached K/V in relevance order
+ * and move K to its new contiguous positions by one more rotary rotation
+ * (Sec. 4.3, Eq. 6-7), attend from the probe tokens to each probe's prefix of
+ * that cache (Eq. 1 and the tree mask of Sec. 4.1), and take the entropy of the
+ * probe's next-token distribution with the threshold rule (Eq. 2).
+ *
+ * Conventions shared by every call
+ *  - Every function returns 0 (ADAPSHOT_OK) or a negative ADAPSHOT_E* code.
+ *    Host-side argument checks happen before any launch; on error nothing is
+ *    enqueued.  Nothing aborts, traps or throws.
+ *  - Structs and `probe_nshots` are HOST memory, read during the call only.
+ *    Every other pointer is a DEVICE pointer owned by the caller, 16-byte
+ *    aligned, valid until the enqueued work has finished.  The library
+ *    allocates no device memory; scratch comes from the caller's `ws`
+ *    (size from the matching *_workspace_bytes function, 256-byte aligned).
+ *  - Work is enqueued asynchronously on `stream` (a cudaStream_t passed as
+ *    void*; NULL = the legacy default stream).  Calls are thread-compatible.
+ *  - `status` is a device int32 the caller zeroes once; kernels only ever
+ *    store a non-zero ADAPSHOT_E* code into it (capacity overflow, bad shot
+ *    id, a pipeline wait that ran out).  The offending unit of work is
+ *    skipped; no out-of-bounds access is made.  Read it after synchronising.
+ *  - Layout names: B queries, k selected shots, P nested probes, T_q probe
+ *    tokens, Hq / Hkv query / KV heads, G = Hq / Hkv, d = head_dim,
+ *    nl = layer_end - layer_begin layers handled by one call.
+ */
+#ifndef ADAPSHOT_H_
+#define ADAPSHOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define ADAPSHOT_API __attribute__((visibility("default")))
+#else
+#define ADAPSHOT_API
+#endif
+
+#define ADAPSHOT_OK            0
+#define ADAPSHOT_EINVAL       -1   /* null pointer, non-positive size, bad flag    */
+#define ADAPSHOT_ESHAPE       -2   /* head_dim, head ratio, probe list, k > N ...  */
+#define ADAPSHOT_EALIGN       -3   /* pointer not 16-byte aligned                  */
+#define ADAPSHOT_ECAPACITY    -4   /* ctx_cap / workspace / static scratch too small */
+#define ADAPSHOT_EUNSUPPORTED -5   /* dtype / mode this build has no kernel for    */
+#define ADAPSHOT_ECUDA        -6   /* a CUDA runtime or driver call failed         */
+#define ADAPSHOT_EINDEX       -7   /* device saw a shot id outside 0..n_shots-1    */
+#define ADAPSHOT_ETIMEOUT     -8   /* device pipeline wait exceeded its limit      */
+
+#define ADAPSHOT_F32   0
+#define ADAPSHOT_BF16  1
+
+/* Model shape (Sec. 4.2: L layers, H heads; grouped-query mapping h -> h / G). */
+typedef struct adapshot_model {
+  int32_t n_layers;       /* layers held by the pool                              */
+  int32_t n_q_heads;      /* Hq                                                   */
+  int32_t n_kv_heads;     /* Hkv, divides Hq                                      */
+  int32_t head_dim;       /* d: 64 or 128                                         */
+  int32_t dtype;          /* storage of pool / ctx / q / out: ADAPSHOT_F32 | BF16 */
+  int32_t k_pos_mode;     /* 0: pool K carries no position (angle (o+t) theta);
+                             1: pool K was rotated at its shot-local position t
+                                (Sec. 4.3: prefilled alone from 0), angle o theta */
+  double  rope_base;      /* theta_i = rope_base^(-2i/d)  (text after Eq. 6)      */
+  float   softmax_scale;  /* 0 => 1/sqrt(d)  (Eq. 5 scaling)                      */
+  int32_t reserved;
+} adapshot_model_t;
+
+/* Global cache pool (Sec. 4.2, Eq. 3), token-major so that one shot's block of
+ * one layer is a single contiguous run:
+ *   k, v : [n_layers][pool_tokens][Hkv][d]   (dtype of the model)
+ *   shot i owns tokens shot_off[i] .. shot_off[i+1]-1 (lengths >= 1)
+ *   emb  : fp32 [n_shots][emb_dim] shot embeddings for the relevance ranking   */
+typedef struct adapshot_pool {
+  int32_t        n_shots;
+  int32_t        emb_dim;
+  int64_t        pool_tokens;
+  const int64_t* shot_off;   /* device, [n_shots + 1], ascending, shot_off[0] = 0 */
+  const void*    k;          /* device */
+  const void*    v;          /* device */
+  const float*   emb;        /* device */
+} adapshot_pool_t;
+
+/* ---- Step 1: relevance ranking and top-k (Sec. 4.1 ranking; Sec. 4.2 "rank in
+ * descending order and select the top k").  score[b][i] = cosine(q_emb[b],
+ * emb[i]) with fp64 accumulation of the fp32 products (0 if either norm is 0);
+ * sel_idx[b][r] = id of the r-th most relevant shot, equal scores ordered by
+ * the lower id.  Nested probes use prefixes of sel_idx.
+ *   q_emb [B][emb_dim] fp32; sel_idx [B][k] int32 out; sel_score [B][k] fp32 out
+ *   or NULL.  Needs 1 <= k <= n_shots.  Scores are compared in fp64.            */
+ADAPSHOT_API size_t adapshot_select_workspace_bytes(int32_t n_shots, int32_t B, int32_t k);
+ADAPSHOT_API int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, int32_t B, int32_t k,
+                    int32_t* sel_idx, float* sel_score,
+                    void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* ---- Step 2: KV-level concatenation with position re-encoding (Sec. 4.3,
+ * Eq. 7; offsets follow the two-shot example: a shot placed after r others
+ * starts at the sum of their lengths).
+ *   ctx_off[b][r] = sum_{r'<r} T_{sel_idx[b][r']}, r = 0..k      (int64 out)
+ *   v_ctx[b][l][o+t][h][:] = v_pool[layer_begin+l][shot_off[s]+t][h][:]  (bit copy)
+ *   k_ctx[b][l][o+t][h][:] = Rot(k_pool[...], Delta theta), o = ctx_off[b][r],
+ *   s = sel_idx[b][r], Delta = o+t (k_pos_mode 0) or o (k_pos_mode 1), with
+ *   Rot(x)_i = x_i cos - x_{i+d/2} sin, Rot(x)_{i+d/2} = x_{i+d/2} cos + x_i sin
+ *   (Eq. 6, half-split rotate_half).  Angles are formed in fp64, the rotation in
+ *   fp32, bf16 results are rounded to nearest-even.
+ *   k_ctx, v_ctx : [B][nl][ctx_cap][Hkv][d]; both NULL => only ctx_off is written.
+ *   Rows L .. min(roundup(L,128), ctx_cap)-1 of every (b, l) are zero-filled so
+ *   that the attention kernel can read whole 128-token tiles.
+ *   Device-detected: L > ctx_cap -> ADAPSHOT_ECAPACITY (tokens beyond the
+ *   capacity are dropped); shot id out of range -> ADAPSHOT_EINDEX (the shot
+ *   counts as length 0).  sel_idx need not come from adapshot_select.           */
+ADAPSHOT_API int adapshot_assemble_kv(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                         const int32_t* sel_idx, int32_t B, int32_t k,
+                         int32_t layer_begin, int32_t layer_end,
+                         void* k_ctx, void* v_ctx, int64_t ctx_cap,
+                         int64_t* ctx_off, uint32_t flags,
+                         int32_t* status, void* stream);
+
+/* ---- Step 3: probe attention over the reused cache (Eq. 1; tree mask of
+ * Sec. 4.1: probe j sees the first probe_nshots[j] shots, i.e. context tokens
+ * 0 .. L_j-1 with L_j = ctx_off[b][probe_nshots[j]], and causally its own T_q
+ * tokens, which sit at positions L_j .. L_j+T_q-1).  For row t and query head h
+ * (KV head h / G): q' = Rot(q, (L_j+t) theta); keys = k_ctx[0..L_j) followed by
+ * Rot(kq[t'], (L_j+t') theta), t' <= t; values = v_ctx[0..L_j) followed by
+ * vq[t' <= t]; out = softmax(q' . keys * scale) . values.
+ *   q   : [B][nl][P][T_q][Hq][d]   un-rotated   (bf16)
+ *   kq,vq: [B][nl][P][T_q][Hkv][d] un-rotated   (bf16)
+ *   out : [B][nl][P][T_q][Hq][d]   (bf16);  lse [B][nl][P][Hq][T_q] fp32 natural-log
+ *         log-sum-exp of the scaled scores, or NULL
+ *   probe_nshots : HOST int32 [P], strictly ascending, 1 <= n_j <= k
+ *   k_ctx, v_ctx, ctx_cap, ctx_off: as written by adapshot_assemble_kv for the
+ *   same B, k and layer range (ctx_cap a multiple of 8).
+ * bf16 tensor-core kernel (tcgen05, fp32 accumulation, split over the context
+ * with a log-sum-exp merge); model->dtype must be ADAPSHOT_BF16.                */
+ADAPSHOT_API size_t adapshot_attn_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
+                                     int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap);
+ADAPSHOT_API int adapshot_query_attn(const adapshot_model_t* model,
+                        const void* k_ctx, const void* v_ctx, int64_t ctx_cap,
+                        const int64_t* ctx_off, int32_t B, int32_t k,
+                        const int32_t* probe_nshots, int32_t P,
+                        const void* q, const void* kq, const void* vq, int32_t Tq,
+                        int32_t layer_begin, int32_t layer_end,
+                        void* out, float* lse, uint32_t flags,
+                        void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* ---- Step 4: confidence probe (Eq. 2 over the whole vocabulary, natural log)
+ * and the threshold rule that follows it.
+ *   H[r] = -sum_v p_v ln p_v, p = softmax(logits[r][0..V))          (fp32 out)
+ *   first_ok[g] = smallest j in 0..rows_per_group-1 with
+ *                 H[g*rows_per_group + j] <= tau, else -1   (int32 out, or NULL)
+ *   logits [R][row_stride] fp32 or bf16 (dtype), row_stride in elements, rows
+ *   16-byte aligned; one pass with a running maximum, fp32 accumulation.        */
+ADAPSHOT_API size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V);
+ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V, int64_t row_stride,
+                     float* H, float tau, int32_t rows_per_group, int32_t* first_ok,
+                     void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+ADAPSHOT_API const char* adapshot_strerror(int code);
+ADAPSHOT_API int adapshot_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAPSHOT_H_ */

@@ -1,0 +1,169 @@
+"""ctypes binding of libadapshot.so: same names as the C ABI, marshalling only.
+
+Every step of the path runs inside the CUDA library.  Importing this module
+raises if the library has not been built: there is no CPU fallback.
+Tensors are torch CUDA tensors used as device memory; the current torch CUDA
+stream is passed to every call.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadapshot.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2605_03644_b200.build` "
+        "(the CUDA library is the only implementation; there is no fallback)")
+lib = C.CDLL(_LIB_PATH)
+
+OK, EINVAL, ESHAPE, EALIGN, ECAPACITY, EUNSUPPORTED, ECUDA, EINDEX, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7, -8
+F32, BF16 = 0, 1
+
+EXPORTS = [
+    "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",
+    "adapshot_attn_workspace_bytes", "adapshot_query_attn",
+    "adapshot_entropy_workspace_bytes", "adapshot_entropy",
+    "adapshot_strerror", "adapshot_version",
+]
+
+
+class ModelT(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("dtype", C.c_int32), ("k_pos_mode", C.c_int32),
+                ("rope_base", C.c_double), ("softmax_scale", C.c_float), ("reserved", C.c_int32)]
+
+
+class PoolT(C.Structure):
+    _fields_ = [("n_shots", C.c_int32), ("emb_dim", C.c_int32), ("pool_tokens", C.c_int64),
+                ("shot_off", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("emb", C.c_void_p)]
+
+
+def _sig(name, restype, argtypes):
+    fn = getattr(lib, name)
+    fn.restype = restype
+    fn.argtypes = argtypes
+    return fn
+
+
+_vp, _i32, _i64, _sz, _u32, _f = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t, C.c_uint32, C.c_float
+_select_ws = _sig("adapshot_select_workspace_bytes", _sz, [_i32, _i32, _i32])
+_select = _sig("adapshot_select", C.c_int, [C.POINTER(PoolT), _vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _vp])
+_assemble = _sig("adapshot_assemble_kv", C.c_int,
+                 [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _i32, _i32, _i32, _i32, _vp, _vp, _i64,
+                  _vp, _u32, _vp, _vp])
+_entropy_ws = _sig("adapshot_entropy_workspace_bytes", _sz, [_i32, _i32])
+_entropy = _sig("adapshot_entropy", C.c_int,
+                [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _sz, _vp, _vp])
+_strerror = _sig("adapshot_strerror", C.c_char_p, [C.c_int])
+_version = _sig("adapshot_version", C.c_int, [])
+_attn_ws = _sig("adapshot_attn_workspace_bytes", _sz, [C.POINTER(ModelT), _i32, _i32, _i32, _i32, _i64])
+_attn = _sig("adapshot_query_attn", C.c_int,
+             [C.POINTER(ModelT), _vp, _vp, _i64, _vp, _i32, _i32, C.POINTER(_i32), _i32,
+              _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+
+
+class AdapshotError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"adapshot error {code}: {adapshot_strerror(code)}")
+
+
+def adapshot_strerror(code: int) -> str:
+    return _strerror(code).decode()
+
+
+def adapshot_version() -> int:
+    return _version()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int):
+    if rc != OK:
+        raise AdapshotError(rc)
+
+
+def make_model(n_layers, n_q_heads, n_kv_heads, head_dim, dtype, rope_base, k_pos_mode=0,
+               softmax_scale=0.0) -> ModelT:
+    dt = {torch.float32: F32, torch.bfloat16: BF16, "fp32": F32, "bf16": BF16}[dtype]
+    return ModelT(n_layers, n_q_heads, n_kv_heads, head_dim, dt, k_pos_mode, float(rope_base),
+                  float(softmax_scale), 0)
+
+
+class Pool:
+    """Holds the device tensors of a pool and the C struct that points at them."""
+
+    def __init__(self, shot_off: torch.Tensor, k: Optional[torch.Tensor], v: Optional[torch.Tensor],
+                 emb: Optional[torch.Tensor]):
+        self.shot_off, self.k, self.v, self.emb = shot_off, k, v, emb
+        n_shots = shot_off.numel() - 1
+        tokens = int(k.shape[1]) if k is not None else 0
+        self.c = PoolT(n_shots, int(emb.shape[1]) if emb is not None else 0, tokens,
+                       _ptr(shot_off), _ptr(k), _ptr(v), _ptr(emb))
+
+
+def adapshot_select_workspace_bytes(n_shots: int, B: int, k: int) -> int:
+    return _select_ws(n_shots, B, k)
+
+
+def adapshot_select(pool: Pool, q_emb: torch.Tensor, k: int, sel_idx: torch.Tensor,
+                    sel_score: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor):
+    B = q_emb.shape[0]
+    _check(_select(C.byref(pool.c), _ptr(q_emb), B, k, _ptr(sel_idx), _ptr(sel_score),
+                   _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_assemble_kv(model: ModelT, pool: Pool, sel_idx: torch.Tensor, layer_begin: int,
+                         layer_end: int, k_ctx: Optional[torch.Tensor], v_ctx: Optional[torch.Tensor],
+                         ctx_cap: int, ctx_off: torch.Tensor, status: torch.Tensor, flags: int = 0):
+    B, k = sel_idx.shape
+    _check(_assemble(C.byref(model), C.byref(pool.c), _ptr(sel_idx), B, k, layer_begin, layer_end,
+                     _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), flags, _ptr(status), _stream()))
+
+
+def adapshot_attn_workspace_bytes(model: ModelT, B: int, P: int, Tq: int, n_layers_in_call: int,
+                                  ctx_cap: int) -> int:
+    return _attn_ws(C.byref(model), B, P, Tq, n_layers_in_call, ctx_cap)
+
+
+def adapshot_query_attn(model: ModelT, k_ctx: torch.Tensor, v_ctx: torch.Tensor, ctx_cap: int,
+                        ctx_off: torch.Tensor, k: int, probe_nshots: Sequence[int],
+                        q: torch.Tensor, kq: torch.Tensor, vq: torch.Tensor,
+                        layer_begin: int, layer_end: int, out: torch.Tensor,
+                        lse: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor,
+                        flags: int = 0):
+    B = q.shape[0]
+    P = len(probe_nshots)
+    Tq = q.shape[3]
+    arr = (_i32 * P)(*[int(x) for x in probe_nshots])
+    _check(_attn(C.byref(model), _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), B, k, arr, P,
+                 _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
+                 flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_entropy_workspace_bytes(R: int, V: int) -> int:
+    return _entropy_ws(R, V)
+
+
+def adapshot_entropy(logits: torch.Tensor, H: torch.Tensor, tau: float, rows_per_group: int,
+                     first_ok: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor):
+    R, V = logits.shape
+    dt = F32 if logits.dtype == torch.float32 else BF16
+    if logits.stride(1) != 1:
+        raise ValueError("logit rows must be contiguous")
+    _check(_entropy(logits.data_ptr(), dt, R, V, logits.stride(0), _ptr(H), tau, rows_per_group,
+                    _ptr(first_ok), _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))

@@ -1,0 +1,58 @@
+// Shared host/device helpers of the adapshot CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "adapshot.h"
+
+#define ADAPSHOT_VERSION_NUMBER 100
+
+#define ADS_CHECK_CUDA(expr)                              \
+  do {                                                    \
+    cudaError_t e__ = (expr);                             \
+    if (e__ != cudaSuccess) return ADAPSHOT_ECUDA;        \
+  } while (0)
+
+static inline bool ads_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t ads_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// A launch failure is reported as ADAPSHOT_ECUDA without clearing anything else.
+static inline int ads_launch_status() {
+  return cudaGetLastError() == cudaSuccess ? ADAPSHOT_OK : ADAPSHOT_ECUDA;
+}
+
+// Device: record an error code once; later codes do not overwrite the first.
+__device__ __forceinline__ void ads_set_status(int32_t* status, int32_t code) {
+  if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Angle p * theta_i formed in fp64 and reduced to [-pi, pi] before the fp32
+// sincos, so that the result keeps fp32 accuracy at positions of 64K and more.
+__device__ __forceinline__ void rope_sincos(double delta, double theta, float* s, float* c) {
+  const double kInv2Pi = 0.15915494309189533577;
+  const double k2PiHi = 6.283185307179586232;
+  const double k2PiLo = 2.449293598294706354e-16;
+  double a = delta * theta;
+  double n = rint(a * kInv2Pi);
+  double r = fma(-n, k2PiHi, a);
+  r = fma(-n, k2PiLo, r);
+  sincosf(static_cast<float>(r), s, c);
+}

@@ -1,0 +1,196 @@
+// Softmax entropy of last-token logits (paper Eq. 2, over the whole vocabulary)
+// and the threshold rule stated after it.
+//
+// One pass: every thread keeps (m, s, t) with s = sum e^{x-m}, t = sum e^{x-m}(x-m)
+// for a running maximum m; states merge exactly (up to rounding) under a change of
+// maximum, and H = ln s - t / s at the end.  Rows are split over several CTAs so a
+// handful of 128K-entry rows still fills the machine; the per-split states go
+// through the caller's workspace and a second, tiny kernel merges them.
+#include <float.h>
+
+#include "common.cuh"
+
+namespace {
+
+struct EntState {
+  float m, s, t;
+};
+
+__device__ __forceinline__ EntState ent_merge(EntState a, EntState b) {
+  float M = fmaxf(a.m, b.m);
+  float ea = __expf(a.m - M), eb = __expf(b.m - M);
+  // a state with s == 0 has seen nothing (or only -inf): it adds nothing
+  float ta = a.s > 0.f ? (a.t + a.s * (a.m - M)) * ea : 0.f;
+  float tb = b.s > 0.f ? (b.t + b.s * (b.m - M)) * eb : 0.f;
+  EntState r;
+  r.m = M;
+  r.s = a.s * ea + b.s * eb;
+  r.t = ta + tb;
+  return r;
+}
+
+template <int N>
+__device__ __forceinline__ void ent_accumulate(EntState& st, const float (&x)[N]) {
+  float vm = x[0];
+#pragma unroll
+  for (int i = 1; i < N; ++i) vm = fmaxf(vm, x[i]);
+  if (vm > st.m) {
+    float e = __expf(st.m - vm);
+    st.t = st.s > 0.f ? (st.t + st.s * (st.m - vm)) * e : 0.f;
+    st.s *= e;
+    st.m = vm;
+  }
+#pragma unroll
+  for (int i = 0; i < N; ++i) {
+    float dlt = x[i] - st.m;
+    float e = __expf(dlt);
+    st.s += e;
+    st.t += e > 0.f ? e * dlt : 0.f;   // -inf logits: e = 0 and the term is 0
+  }
+}
+
+__device__ __forceinline__ EntState ent_warp_reduce(EntState st) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    EntState other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
+    other.t = __shfl_xor_sync(0xffffffffu, st.t, o);
+    st = ent_merge(st, other);
+  }
+  return st;
+}
+
+constexpr int kEntThreads = 256;
+
+// grid (n_split, R).  partial[(r * n_split + s)] = state of slice s of row r.
+template <typename T>
+__global__ void __launch_bounds__(kEntThreads)
+entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride, int slice,
+                       float* __restrict__ partial) {
+  constexpr int kVec = 16 / sizeof(T);
+  const int r = blockIdx.y, sp = blockIdx.x, n_split = gridDim.x;
+  const T* row = logits + (long long)r * row_stride;
+  const int begin = sp * slice;
+  const int end = min(V, begin + slice);
+  EntState st{-FLT_MAX, 0.f, 0.f};
+
+  const int vec_end = begin + ((end - begin) / kVec) * kVec;   // slice is a multiple of kVec
+  for (int i = begin + threadIdx.x * kVec; i < vec_end; i += kEntThreads * kVec) {
+    float x[kVec];
+    uint4 raw = *reinterpret_cast<const uint4*>(row + i);
+    if constexpr (sizeof(T) == 4) {
+      x[0] = __uint_as_float(raw.x); x[1] = __uint_as_float(raw.y);
+      x[2] = __uint_as_float(raw.z); x[3] = __uint_as_float(raw.w);
+    } else {
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
+        x[2 * j] = __uint_as_float(w[j] << 16);
+        x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      }
+    }
+    ent_accumulate(st, x);
+  }
+  for (int i = vec_end + threadIdx.x; i < end; i += kEntThreads) {   // ragged tail of the row
+    float x[1];
+    if constexpr (sizeof(T) == 4) x[0] = row[i];
+    else x[0] = __bfloat162float(row[i]);
+    ent_accumulate(st, x);
+  }
+
+  st = ent_warp_reduce(st);
+  __shared__ EntState sh[kEntThreads / 32];
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = st;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    EntState v = threadIdx.x < kEntThreads / 32 ? sh[threadIdx.x] : EntState{-FLT_MAX, 0.f, 0.f};
+    v = ent_warp_reduce(v);
+    if (threadIdx.x == 0) {
+      float* o = partial + 3ll * ((long long)r * n_split + sp);
+      o[0] = v.m; o[1] = v.s; o[2] = v.t;
+    }
+  }
+}
+
+// One CTA per group of `rows_per_group` rows; warp w merges the splits of rows
+// w, w + n_warps, ...; thread 0 then applies the threshold rule to the group.
+__global__ void __launch_bounds__(256)
+entropy_finish_kernel(const float* __restrict__ partial, int n_split, int R, int rows_per_group,
+                      float tau, float* __restrict__ H, int32_t* __restrict__ first_ok) {
+  extern __shared__ float sh_h[];
+  const int g = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  for (int j = warp; j < rows_per_group; j += n_warps) {
+    const int r = g * rows_per_group + j;
+    if (r >= R) break;
+    EntState st{-FLT_MAX, 0.f, 0.f};
+    for (int s = lane; s < n_split; s += 32) {
+      const float* p = partial + 3ll * ((long long)r * n_split + s);
+      st = ent_merge(st, EntState{p[0], p[1], p[2]});
+    }
+    st = ent_warp_reduce(st);
+    if (lane == 0) {
+      float h = st.s > 0.f ? logf(st.s) - st.t / st.s : 0.f;
+      h = fmaxf(h, 0.f);
+      H[r] = h;
+      sh_h[j] = h;
+    }
+  }
+  __syncthreads();
+  if (first_ok != nullptr && threadIdx.x == 0) {
+    int ok = -1;
+    for (int j = 0; j < rows_per_group && g * rows_per_group + j < R; ++j) {
+      if (sh_h[j] <= tau) { ok = j; break; }
+    }
+    first_ok[g] = ok;
+  }
+}
+
+int ent_splits(int R, int V) {
+  // enough CTAs for about two waves of 148 SMs, each slice at least 4096 entries
+  int want = (2 * 148 + R - 1) / R;
+  int max_by_len = (V + 4095) / 4096;
+  int s = want < max_by_len ? want : max_by_len;
+  return s < 1 ? 1 : s;
+}
+
+}  // namespace
+
+extern "C" size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V) {
+  if (R <= 0 || V <= 0) return 0;
+  return ads_round_up((size_t)R * ent_splits(R, V) * 3 * sizeof(float), 256);
+}
+
+extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V,
+                                int64_t row_stride, float* H, float tau, int32_t rows_per_group,
+                                int32_t* first_ok, void* ws, size_t ws_bytes, int32_t* status,
+                                void* stream) {
+  (void)status;
+  if (logits == nullptr || H == nullptr || ws == nullptr) return ADAPSHOT_EINVAL;
+  if (R <= 0 || V <= 0 || row_stride < V) return ADAPSHOT_EINVAL;
+  if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
+  if (rows_per_group <= 0) rows_per_group = 1;
+  if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
+  if (!ads_aligned16(logits) || !ads_aligned16(ws) || (row_stride * es) % 16 != 0) return ADAPSHOT_EALIGN;
+  if (ws_bytes < adapshot_entropy_workspace_bytes(R, V)) return ADAPSHOT_ECAPACITY;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_split = ent_splits(R, V);
+  const int vec = 16 / (int)es;
+  int slice = (V + n_split - 1) / n_split;
+  slice = (slice + vec - 1) / vec * vec;
+  dim3 grid(n_split, R);
+  float* partial = static_cast<float*>(ws);
+  if (dtype == ADAPSHOT_F32)
+    entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(
+        static_cast<const float*>(logits), V, row_stride, slice, partial);
+  else
+    entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, partial);
+  if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  entropy_finish_kernel<<<R / rows_per_group, 256, rows_per_group * sizeof(float), st>>>(
+      partial, n_split, R, rows_per_group, tau, H, first_ok);
+  return ads_launch_status();
+}

@@ -1,0 +1,245 @@
+// Semantic shot selection (paper Sec. 4.1 ranking, Sec. 4.2 "rank in descending
+// order and select the top k"): cosine of the query embedding against every cached
+// shot embedding, then a block-wide top-k with ties broken by the lower shot id.
+//
+// The ranking must equal that of an fp64 evaluation of the same formula, so the
+// fp32 products (exact in fp64) are accumulated in fp64 and scores are compared in
+// fp64; the table is read once and the kernel stays bandwidth-bound.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kSortCap = 8192;      // candidates one CTA sorts in shared memory
+constexpr int kSortThreads = 1024;
+
+// One warp per pool row i: dots[b][i] = <q_b, e_i> for all b, enorm[i] = |e_i|.
+__global__ void __launch_bounds__(256)
+cosine_dots_kernel(const float* __restrict__ emb, const float* __restrict__ q_emb, int N, int E,
+                   int B, double* __restrict__ dots, double* __restrict__ enorm) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= N) return;
+  const float* e = emb + (long long)row * E;
+  const bool vec_ok = (E & 3) == 0;
+  double nn = 0.0;
+  if (vec_ok) {
+    for (int i = lane * 4; i < E; i += 128) {
+      float4 v = *reinterpret_cast<const float4*>(e + i);
+      nn += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
+    }
+  } else {
+    for (int i = lane; i < E; i += 32) nn += (double)e[i] * e[i];
+  }
+  nn = warp_sum(nn);
+  if (lane == 0) enorm[row] = sqrt(nn);
+  for (int b = 0; b < B; ++b) {
+    const float* q = q_emb + (long long)b * E;
+    double acc = 0.0;
+    if (vec_ok) {
+      for (int i = lane * 4; i < E; i += 128) {
+        float4 v = *reinterpret_cast<const float4*>(e + i);   // L1-resident after the first pass
+        float4 w = __ldg(reinterpret_cast<const float4*>(q + i));
+        acc += (double)v.x * w.x + (double)v.y * w.y + (double)v.z * w.z + (double)v.w * w.w;
+      }
+    } else {
+      for (int i = lane; i < E; i += 32) acc += (double)e[i] * q[i];
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) dots[(long long)b * N + row] = acc;
+  }
+}
+
+// Order-preserving map of an fp64 score to an unsigned key; larger score -> SMALLER
+// key so that an ascending sort on (key, id) lists the most relevant shot first and
+// equal scores by ascending id.
+__device__ __forceinline__ unsigned long long desc_key(double s) {
+  unsigned long long u = (unsigned long long)__double_as_longlong(s);
+  u = (u >> 63) ? ~u : (u | 0x8000000000000000ull);   // ascending in s
+  return ~u;
+}
+__device__ __forceinline__ double key_score(unsigned long long k) {
+  unsigned long long u = ~k;
+  u = (u >> 63) ? (u & 0x7fffffffffffffffull) : ~u;
+  return __longlong_as_double((long long)u);
+}
+
+__device__ __forceinline__ bool pair_less(unsigned long long ka, int ia, unsigned long long kb, int ib) {
+  return ka < kb || (ka == kb && ia < ib);
+}
+
+// grid (n_chunks, B).  Sorts candidates [chunk*kSortCap, ...) of query b and writes
+// the first min(k, n_in_chunk) of them to out_key/out_id at [b][chunk*k + r].
+// Round 0 builds the candidates from dots / norms (in_key == nullptr).
+__global__ void __launch_bounds__(kSortThreads)
+topk_sort_kernel(const double* __restrict__ dots, const double* __restrict__ enorm,
+                 const float* __restrict__ q_emb, int E,
+                 const unsigned long long* __restrict__ in_key, const int* __restrict__ in_id,
+                 int n_in, int in_stride, int k, unsigned long long* __restrict__ out_key,
+                 int* __restrict__ out_id,
+                 int out_stride, int32_t* __restrict__ final_idx, float* __restrict__ final_score) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
+  int* ids = reinterpret_cast<int*>(keys + kSortCap);
+  __shared__ double red[kSortThreads / 32];
+  __shared__ double qnorm_sh;
+
+  const int b = blockIdx.y, chunk = blockIdx.x;
+  const int begin = chunk * kSortCap;
+  const int n = min(kSortCap, n_in - begin);
+  int n_pow2 = 1;
+  while (n_pow2 < n) n_pow2 <<= 1;
+
+  if (in_key == nullptr) {
+    // |q_b| in fp64, once per CTA
+    const float* q = q_emb + (long long)b * E;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < E; i += kSortThreads) acc += (double)q[i] * q[i];
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      double v = red[threadIdx.x];
+      v = warp_sum(v);
+      if (threadIdx.x == 0) qnorm_sh = sqrt(v);
+    }
+    __syncthreads();
+    const double qn = qnorm_sh;
+    for (int i = threadIdx.x; i < n_pow2; i += kSortThreads) {
+      if (i < n) {
+        double den = qn * enorm[begin + i];
+        double s = den > 0.0 ? dots[(long long)b * in_stride + begin + i] / den : 0.0;
+        keys[i] = desc_key(s);
+        ids[i] = begin + i;
+      } else {
+        keys[i] = ~0ull;             // padding sorts last
+        ids[i] = 0x7fffffff;
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < n_pow2; i += kSortThreads) {
+      if (i < n) {
+        keys[i] = in_key[(long long)b * in_stride + begin + i];
+        ids[i] = in_id[(long long)b * in_stride + begin + i];
+      } else {
+        keys[i] = ~0ull;
+        ids[i] = 0x7fffffff;
+      }
+    }
+  }
+  __syncthreads();
+
+  // bitonic sort, ascending on (key, id); ids are unique so the order is total
+  for (int size = 2; size <= n_pow2; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < (n_pow2 >> 1); t += kSortThreads) {
+        int lo = 2 * t - (t & (stride - 1));
+        int hi = lo + stride;
+        bool up = (lo & size) == 0;
+        unsigned long long ka = keys[lo], kb = keys[hi];
+        int ia = ids[lo], ib = ids[hi];
+        bool swap = up ? pair_less(kb, ib, ka, ia) : pair_less(ka, ia, kb, ib);
+        if (swap) {
+          keys[lo] = kb; keys[hi] = ka;
+          ids[lo] = ib; ids[hi] = ia;
+        }
+      }
+      __syncthreads();
+    }
+  }
+
+  const int n_out = min(k, n);
+  if (final_idx != nullptr) {
+    for (int r = threadIdx.x; r < n_out; r += kSortThreads) {
+      final_idx[(long long)b * k + r] = ids[r];
+      if (final_score != nullptr) final_score[(long long)b * k + r] = (float)key_score(keys[r]);
+    }
+  } else {
+    for (int r = threadIdx.x; r < n_out; r += kSortThreads) {
+      out_key[(long long)b * out_stride + chunk * k + r] = keys[r];
+      out_id[(long long)b * out_stride + chunk * k + r] = ids[r];
+    }
+  }
+}
+
+size_t sel_cand_entries(int n_shots, int k) {
+  if (n_shots <= kSortCap) return 0;
+  size_t chunks = ((size_t)n_shots + kSortCap - 1) / kSortCap;
+  return chunks * (size_t)k;
+}
+
+}  // namespace
+
+extern "C" size_t adapshot_select_workspace_bytes(int32_t n_shots, int32_t B, int32_t k) {
+  if (n_shots <= 0 || B <= 0 || k <= 0) return 0;
+  size_t bytes = ads_round_up((size_t)B * n_shots * sizeof(double), 256);   // dots
+  bytes += ads_round_up((size_t)n_shots * sizeof(double), 256);             // |e_i|
+  size_t cand = sel_cand_entries(n_shots, k);
+  // two ping-pong candidate lists of (key, id)
+  bytes += 2 * (ads_round_up((size_t)B * cand * 8, 256) + ads_round_up((size_t)B * cand * 4, 256));
+  return bytes;
+}
+
+extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, int32_t B, int32_t k,
+                               int32_t* sel_idx, float* sel_score, void* ws, size_t ws_bytes,
+                               int32_t* status, void* stream) {
+  (void)status;
+  if (pool == nullptr || q_emb == nullptr || sel_idx == nullptr || ws == nullptr) return ADAPSHOT_EINVAL;
+  if (pool->emb == nullptr || pool->n_shots <= 0 || pool->emb_dim <= 0 || B <= 0) return ADAPSHOT_EINVAL;
+  const int N = pool->n_shots, E = pool->emb_dim;
+  if (k < 1 || k > N) return ADAPSHOT_ESHAPE;
+  if (N > kSortCap && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
+  if (!ads_aligned16(pool->emb) || !ads_aligned16(q_emb) || !ads_aligned16(ws)) return ADAPSHOT_EALIGN;
+  if (ws_bytes < adapshot_select_workspace_bytes(N, B, k)) return ADAPSHOT_ECAPACITY;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* p = static_cast<unsigned char*>(ws);
+  double* dots = reinterpret_cast<double*>(p);
+  p += ads_round_up((size_t)B * N * sizeof(double), 256);
+  double* enorm = reinterpret_cast<double*>(p);
+  p += ads_round_up((size_t)N * sizeof(double), 256);
+  const size_t cand = sel_cand_entries(N, k);
+  unsigned long long* ckey[2];
+  int* cid[2];
+  for (int i = 0; i < 2; ++i) {
+    ckey[i] = reinterpret_cast<unsigned long long*>(p);
+    p += ads_round_up((size_t)B * cand * 8, 256);
+    cid[i] = reinterpret_cast<int*>(p);
+    p += ads_round_up((size_t)B * cand * 4, 256);
+  }
+
+  const int warps_per_block = 8;
+  cosine_dots_kernel<<<(N + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+      pool->emb, q_emb, N, E, B, dots, enorm);
+  if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+
+  const size_t smem = (size_t)kSortCap * (8 + 4);
+  static bool attr_set = false;   // same value every time: a benign race
+  if (!attr_set) {
+    ADS_CHECK_CUDA(cudaFuncSetAttribute(topk_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_set = true;
+  }
+
+  int n_in = N, in_stride = N;
+  int round = 0;
+  const unsigned long long* in_key = nullptr;
+  const int* in_id = nullptr;
+  while (true) {
+    const int chunks = (n_in + kSortCap - 1) / kSortCap;
+    const bool last = chunks == 1;
+    dim3 grid(chunks, B);
+    const int out_stride = chunks * k;
+    topk_sort_kernel<<<grid, kSortThreads, smem, st>>>(
+        dots, enorm, q_emb, E, in_key, in_id, n_in, in_stride, k, ckey[round & 1], cid[round & 1], out_stride,
+        last ? sel_idx : nullptr, last ? sel_score : nullptr);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+    if (last) break;
+    in_key = ckey[round & 1];
+    in_id = cid[round & 1];
+    // every chunk but possibly the last holds >= k candidates (k <= kSortCap / 2)
+    const int last_n = n_in - (chunks - 1) * kSortCap;
+    n_in = (chunks - 1) * k + (last_n < k ? last_n : k);
+    in_stride = out_stride;
+    ++round;
+  }
+  return ADAPSHOT_OK;
+}

@@ -1,0 +1,78 @@
+"""CPU checks of the boundary: the library loads, exports what the header declares,
+and rejects bad arguments on the host before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def ab():
+    from paper_2605_03644_b200 import build
+    build.build()
+    from paper_2605_03644_b200 import binding
+    return binding
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "adapshot.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(adapshot_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(ab):
+    names = _declared()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(ab.lib, n), f"{n} declared in adapshot.h but not exported"
+    assert sorted(ab.EXPORTS) == sorted(n for n in names if not n.endswith("_t"))
+
+
+def test_version_and_strerror(ab):
+    assert ab.adapshot_version() >= 100
+    assert ab.adapshot_strerror(0) == "ok"
+    for code in range(-8, 0):
+        assert "unknown" not in ab.adapshot_strerror(code)
+    assert "unknown" in ab.adapshot_strerror(-99)
+
+
+def test_workspace_sizes(ab):
+    assert ab.adapshot_select_workspace_bytes(0, 1, 1) == 0
+    assert ab.adapshot_select_workspace_bytes(2048, 1, 128) >= 2048 * 8 * 2
+    assert ab.adapshot_entropy_workspace_bytes(4, 32000) >= 4 * 12
+    assert ab.adapshot_entropy_workspace_bytes(4, 32000) % 256 == 0
+
+
+def test_host_side_argument_checks_launch_nothing(ab):
+    # all of these return before any CUDA call, so they run without a device
+    pool = ab.PoolT(16, 8, 100, 0x1000, 0x1000, 0x1000, 0x1000)
+    model = ab.make_model(1, 4, 1, 64, "fp32", 1e4)
+    fake = C.c_void_p(0x1000)
+    sel = ab.lib.adapshot_select
+    assert sel(C.byref(pool), None, 1, 4, fake, None, fake, 1 << 20, None, None) == ab.EINVAL
+    assert sel(C.byref(pool), fake, 1, 17, fake, None, fake, 1 << 20, None, None) == ab.ESHAPE   # k > N
+    assert sel(C.byref(pool), fake, 1, 0, fake, None, fake, 1 << 20, None, None) == ab.ESHAPE
+    assert sel(C.byref(pool), C.c_void_p(0x1004), 1, 4, fake, None, fake, 1 << 20, None, None) == ab.EALIGN
+    assert sel(C.byref(pool), fake, 1, 4, fake, None, fake, 16, None, None) == ab.ECAPACITY
+    asm = ab.lib.adapshot_assemble_kv
+    args = lambda m, **kw: [C.byref(m), C.byref(pool), fake, 1, kw.get("k", 4), kw.get("lb", 0), kw.get("le", 1),
+                            kw.get("kc", fake), kw.get("vc", fake), kw.get("cap", 256), fake, kw.get("flags", 0), None, None]
+    assert asm(*args(model, k=17)) == ab.ESHAPE
+    assert asm(*args(model, le=2)) == ab.ESHAPE                       # layer range outside the model
+    assert asm(*args(model, flags=1)) == ab.EINVAL
+    assert asm(*args(model, vc=None)) == ab.EINVAL                    # only one of k_ctx / v_ctx
+    assert asm(*args(model, kc=C.c_void_p(0x1008))) == ab.EALIGN
+    bad = ab.make_model(1, 4, 1, 96, "fp32", 1e4)
+    assert asm(*args(bad)) == ab.ESHAPE                               # head_dim not 64 / 128
+    bad = ab.make_model(1, 5, 2, 64, "fp32", 1e4)
+    assert asm(*args(bad)) == ab.ESHAPE                               # Hq % Hkv != 0
+    ent = ab.lib.adapshot_entropy
+    assert ent(None, 0, 1, 8, 8, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EINVAL
+    assert ent(fake, 2, 1, 8, 8, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EUNSUPPORTED
+    assert ent(fake, 0, 3, 8, 8, fake, 0.5, 2, None, fake, 1 << 20, None, None) == ab.ESHAPE     # R % P
+    assert ent(fake, 0, 1, 8, 4, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EINVAL     # stride < V
+    assert ent(fake, 1, 2, 8, 9, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EALIGN     # bf16 row 18 B
+    assert ent(fake, 0, 1, 8, 8, fake, 0.5, 1, None, fake, 0, None, None) == ab.ECAPACITY

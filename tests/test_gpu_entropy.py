@@ -1,0 +1,81 @@
+"""adapshot_entropy vs the fp64 oracle: relative error <= 1e-4."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import adapshot_oracle as orc
+from paper_2605_03644_b200 import workloads as wl
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+REL_TOL = 1e-4
+
+
+def _check(ab, logits, tau=None, P=1):
+    H, fo, st = hp.run_entropy(ab, logits.cuda(), 0.0 if tau is None else tau, P)
+    want = orc.entropy(hp.f64(logits))
+    got = H.cpu().numpy().astype(np.float64)
+    assert st == 0
+    rel = np.abs(got - want) / np.maximum(np.abs(want), 1e-3)
+    assert rel.max() <= REL_TOL, rel.max()
+    if tau is not None:
+        # keep the threshold decision away from rounding: every |H - tau| must be clear
+        assert np.abs(want - tau).min() > 1e-3 * max(tau, 1.0)
+        assert np.array_equal(fo.cpu().numpy(), orc.first_ok(want, tau, P))
+    return got
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3"])
+def test_entropy_on_config_logits(name):
+    ab = hp.gpu_binding()
+    w = wl.CONFIGS[name]
+    P = len(w.probes)
+    g = torch.Generator().manual_seed(w.seed)
+    ldt = torch.float32 if w.logits_dtype == "fp32" else torch.bfloat16
+    logits = (torch.randn(w.batch * P, w.vocab, generator=g) * w.logits_std).to(ldt)
+    _check(ab, logits)
+
+
+def test_entropy_cfg5_probe_rows_bf16():
+    ab = hp.gpu_binding()
+    g = torch.Generator().manual_seed(9)
+    # 3 queries x 7 nested probes at the full vocabulary; sharper rows for later probes
+    sharp = torch.tensor([0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]).repeat(3)[:, None]
+    logits = (torch.randn(21, 128256, generator=g) * sharp).to(torch.bfloat16)
+    want = orc.entropy(hp.f64(logits))
+    tau = float((want.reshape(3, 7)[:, 3] + want.reshape(3, 7)[:, 4]).mean() / 2)
+    _check(ab, logits, tau=tau, P=7)
+
+
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 9, 1023, 4097, 50001])
+@pytest.mark.parametrize("dt", [torch.float32, torch.bfloat16])
+def test_entropy_ragged_vocab(V, dt):
+    ab = hp.gpu_binding()
+    g = torch.Generator().manual_seed(V)
+    stride = (V + 7) // 8 * 8                      # rows must start on 16 bytes
+    buf = (torch.randn(5, stride, generator=g) * 3).to(dt).cuda()
+    H, _, st = hp.run_entropy(ab, buf[:, :V], 0.0, 1, want_first=False)
+    want = orc.entropy(hp.f64(buf[:, :V]))
+    assert st == 0
+    assert np.all(np.abs(H.cpu().numpy() - want) <= REL_TOL * np.maximum(want, 1e-3) + 1e-7)
+
+
+def test_entropy_closed_forms_and_threshold():
+    ab = hp.gpu_binding()
+    V = 32000
+    x = torch.zeros(4, V)
+    x[1, 5] = 200.0                                # one dominant logit -> 0
+    x[2, :10] = 1.5; x[2, 10:] = -0.5              # two-level row
+    x[3] = -1e4; x[3, :2] = 0.0                    # two equal survivors -> ln 2
+    x[3, 100:200] = float("-inf")
+    got = _check(ab, x)
+    assert abs(got[0] - math.log(V)) < 1e-4 * math.log(V)
+    assert got[1] < 1e-6 and abs(got[3] - math.log(2)) < 1e-5
+    H, fo, _ = hp.run_entropy(ab, x.cuda(), 1.0, 2)
+    assert fo.tolist() == [1, 1]                   # groups (uniform, peaked) and (two-level, ln 2)
+    H, fo, _ = hp.run_entropy(ab, x.cuda(), 1e-9, 4)
+    assert fo.tolist() == [1]
+    H, fo, _ = hp.run_entropy(ab, x[:1].cuda(), 1.0, 1)
+    assert fo.tolist() == [-1]

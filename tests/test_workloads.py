@@ -1,0 +1,34 @@
+"""The seeded generators are deterministic and have the stated shapes."""
+import numpy as np
+import torch
+
+from paper_2605_03644_b200 import workloads as wl
+
+
+def test_lengths_follow_the_recipes():
+    for name, w in wl.CONFIGS.items():
+        t = wl.shot_lengths(w)
+        assert np.array_equal(t, wl.shot_lengths(w))
+        assert t.min() >= w.len_lo and t.max() <= w.len_hi
+        if w.n_shots:
+            assert len(t) == w.n_shots
+        else:
+            assert t.sum() >= w.pool_token_target > t[:-1].sum()
+    t5 = wl.shot_lengths(wl.CONFIGS["cfg5"])
+    assert 110 <= np.median(t5) <= 130
+
+
+def test_small_pool_and_queries_are_reproducible():
+    w = wl.CONFIGS["cfg1"]
+    a, b = wl.make_pool(w), wl.make_pool(w)
+    assert torch.equal(a["k"], b["k"]) and torch.equal(a["emb"], b["emb"])
+    assert a["k"].shape == (1, 64 * 32, 1, 64) and a["k"].dtype == torch.float32
+    assert torch.allclose(a["emb"].norm(dim=1), torch.ones(64), atol=1e-6)
+    q = wl.make_queries(w)
+    assert q["q"].shape == (1, 1, 1, 16, 4, 64) and q["logits"].shape == (1, 1024)
+    assert abs(q["logits"].var().item() - 2.0) < 0.3
+    w2 = wl.CONFIGS["cfg2"].scaled(n_shots=32)
+    p2 = wl.make_pool(w2)
+    assert p2["k"].dtype == torch.bfloat16 and p2["pool_tokens"] == int(p2["shot_off"][-1])
+    x = wl.to_f64(p2["k"])
+    assert x.dtype == np.float64 and np.array_equal(x.astype(np.float32), p2["k"].float().numpy())
