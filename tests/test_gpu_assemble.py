@@ -1,5 +1,5 @@
 """adapshot_assemble_kv vs the fp64 oracle: offsets and V bit-exact; fp32 K within
-1e-5 max-abs; bf16 K within one bf16 code point of the rounded oracle value."""
+1e-5 max-abs; bf16 K within half a bf16 step (+1e-5) of the oracle, >= 99 % bit-equal."""
 import numpy as np
 import pytest
 import torch
@@ -28,10 +28,14 @@ def _compare(w, pool, sel_np, kc, vc, off, nl_begin, nl_end, k_pos_mode=0):
             err = (got_k.double() - torch.from_numpy(ok)).abs().max().item()
             assert err <= K_TOL_FP32, err
         else:
-            ref = torch.from_numpy(ok).to(torch.float32).to(torch.bfloat16)
-            ulp = hp.bf16_ulp_diff(got_k, ref)
-            assert ulp.max().item() <= 1
-            assert (ulp == 0).float().mean().item() >= 0.99
+            # bf16 store: one round-to-nearest-even of the fp32 rotation, so the error is
+            # at most half a bf16 step (2^-8 relative) plus the fp32 slack; and nearly
+            # every element must equal the rounded oracle value bit for bit
+            want = torch.from_numpy(ok)
+            err = (got_k.double() - want).abs()
+            assert (err <= want.abs() * 2.0 ** -8 + K_TOL_FP32).all(), err.max().item()
+            ref = want.to(torch.float32).to(torch.bfloat16)
+            assert (hp.bf16_ulp_diff(got_k, ref) == 0).float().mean().item() >= 0.99
         # zero padding up to the 128-token tile edge, untouched canary after it
         pad_end = min((L + 127) // 128 * 128, kc.shape[2])
         assert (kc[b, :, L:pad_end] == 0).all() and (vc[b, :, L:pad_end] == 0).all()
