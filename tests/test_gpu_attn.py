@@ -1,0 +1,106 @@
+"""adapshot_query_attn vs the fp64 oracle: bf16 output within max-abs 2e-2 and
+mean-abs 2e-3 (the stated tolerance); log-sum-exp within 2e-3."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adapshot_oracle as orc
+from paper_2605_03644_b200 import workloads as wl
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+MAX_ABS, MEAN_ABS, LSE_ABS = 2e-2, 2e-3, 2e-3
+
+
+def _oracle_ctx(w, pool, sel_np, nl):
+    """Assembled cache from the oracle, rounded once to the bf16 storage format."""
+    kp, vp = hp.f64(pool["k"][:nl]), hp.f64(pool["v"][:nl])
+    outs = []
+    for b in range(sel_np.shape[0]):
+        ok, ov, off = orc.assemble_kv(kp, vp, pool["shot_off"], sel_np[b], w.rope_base)
+        outs.append((torch.from_numpy(ok).to(torch.bfloat16), torch.from_numpy(ov).to(torch.bfloat16), off))
+    return outs
+
+
+def _run_case(w, sel_np, probes, nl, flags=0, cap_extra=37):
+    ab = hp.gpu_binding()
+    w = w.scaled(probes=tuple(probes))
+    pool = wl.make_pool(w, n_layers=nl)
+    qs = wl.make_queries(w, n_layers=nl)
+    if w.dtype == "fp32":        # the attention kernel is bf16: round the inputs once, for both sides
+        w = w.scaled(dtype="bf16")
+        for key in ("k", "v"):
+            pool[key] = pool[key].to(torch.bfloat16)
+        for key in ("q", "kq", "vq"):
+            qs[key] = qs[key].to(torch.bfloat16)
+    B, k = sel_np.shape
+    ctxs = _oracle_ctx(w, pool, sel_np, nl)
+    cap = max(int(c[2][-1]) for c in ctxs) + cap_extra
+    kc = torch.zeros((B, nl, cap, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    off = torch.zeros((B, k + 1), dtype=torch.int64)
+    for b, (ok, ov, o) in enumerate(ctxs):
+        L = int(o[-1])
+        kc[b, :, :L], vc[b, :, :L] = ok, ov
+        off[b] = torch.from_numpy(o)
+    model = hp.model_of(ab, w, n_layers=nl)
+    q, kq, vq = qs["q"].cuda(), qs["kq"].cuda(), qs["vq"].cuda()
+    ws_flags = flags
+    out = torch.full_like(q, 9.0)
+    lse = torch.zeros((B, nl, len(probes), w.n_q_heads, w.t_q), dtype=torch.float32, device="cuda")
+    ws = torch.empty(ab.adapshot_attn_workspace_bytes(model, B, len(probes), w.t_q, nl, cap),
+                     dtype=torch.uint8, device="cuda")
+    st = hp.new_status()
+    ab.adapshot_query_attn(model, kc.cuda(), vc.cuda(), cap, off.cuda(), k, list(probes), q, kq, vq, 0, nl,
+                           out, lse, ws, st, flags=ws_flags)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    worst, mean_acc, n = 0.0, 0.0, 0
+    for b in range(B):
+        L_list = [int(off[b, n_j]) for n_j in probes]
+        for l in range(nl):
+            want, want_lse = orc.query_attn(hp.f64(qs["q"][b, l]), hp.f64(qs["kq"][b, l]), hp.f64(qs["vq"][b, l]),
+                                            hp.f64(kc[b, l]), hp.f64(vc[b, l]), L_list, w.rope_base)
+            err = np.abs(out[b, l].cpu().double().numpy() - want)
+            worst = max(worst, err.max()); mean_acc += err.sum(); n += err.size
+            assert np.abs(lse[b, l].cpu().double().numpy() - want_lse).max() <= LSE_ABS
+    assert worst <= MAX_ABS, worst
+    assert mean_acc / n <= MEAN_ABS, mean_acc / n
+    return worst, mean_acc / n
+
+
+def test_cfg1_attention():
+    w = wl.CONFIGS["cfg1"]
+    pool = wl.make_pool(w)
+    qs = wl.make_queries(w)
+    sel, _ = orc.select_topk(hp.f64(qs["q_emb"]), hp.f64(pool["emb"]), w.k)
+    _run_case(w, sel, [8], 1)
+
+
+@pytest.mark.parametrize("flags", [0, 8])
+def test_8b_shape_ragged_probes_and_chunks(flags):
+    # several 128-key tiles, a ragged last tile, nested probes, two layers, two queries
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=64, len_lo=30, len_hi=90, batch=2, k=40, t_q=40, seed=21)
+    rng = np.random.default_rng(1)
+    sel = np.stack([rng.permutation(64)[:40], rng.permutation(64)[:40]]).astype(np.int32)
+    _run_case(w, sel, [3, 17, 40], 2, flags=flags)
+
+
+def test_tq_longer_than_a_key_tile_and_g8():
+    # T_q = 150 > 128: two own-key tiles with the causal diagonal; G = 8 rows per token
+    w = wl.CONFIGS["cfg4"].scaled(n_shots=20, len_lo=10, len_hi=40, batch=1, k=9, t_q=150, n_q_heads=16,
+                                  n_kv_heads=2, pool_token_target=0, seed=22)
+    sel = np.arange(9, dtype=np.int32)[None, ::-1].copy()
+    _run_case(w, sel, [2, 9], 1)
+
+
+def test_single_token_probe_and_tiny_context():
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=8, len_lo=1, len_hi=3, batch=1, k=2, t_q=1, seed=23)
+    _run_case(w, np.array([[5, 1]], dtype=np.int32), [1, 2], 1)
+
+
+def test_head_dim_64_bf16_many_tiles():
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=32, len_lo=50, len_hi=120, batch=1, k=20, t_q=33, head_dim=64,
+                                  n_q_heads=6, n_kv_heads=3, seed=24)
+    sel = np.random.default_rng(2).permutation(32)[:20].astype(np.int32)[None]
+    _run_case(w, sel, [20], 1)
