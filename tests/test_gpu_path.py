@@ -1,0 +1,76 @@
+"""The whole hot path (select -> assemble -> attention -> entropy) through the host
+driver against the oracle chain, at the tolerances stated for each step."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adapshot_oracle as orc
+from paper_2605_03644_b200 import workloads as wl
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_path(w, pool, qs, nl, tau):
+    """Oracle results for every query of the workload (K' kept in fp64, never rounded)."""
+    sel, _ = orc.select_topk(hp.f64(qs["q_emb"]), hp.f64(pool["emb"]), w.k)
+    off = orc.plan_offsets(sel, pool["shot_off"])
+    kp, vp = hp.f64(pool["k"][:nl]), hp.f64(pool["v"][:nl])
+    outs = []
+    for b in range(w.batch):
+        kc, vc, _ = orc.assemble_kv(kp, vp, pool["shot_off"], sel[b], w.rope_base)
+        L_list = [int(off[b, n]) for n in w.probes]
+        per_layer = [orc.query_attn(hp.f64(qs["q"][b, l]), hp.f64(qs["kq"][b, l]), hp.f64(qs["vq"][b, l]),
+                                    kc[l], vc[l], L_list, w.rope_base)[0] for l in range(nl)]
+        outs.append(np.stack(per_layer))
+    H = orc.entropy(hp.f64(qs["logits"]))
+    return sel, off, np.stack(outs), H, orc.first_ok(H, tau, len(w.probes))
+
+
+def run_gpu_path(w, pool, qs, nl, tau, layers_per_call=None, ctx_cap=None):
+    from paper_2605_03644_b200 import binding as ab
+    from paper_2605_03644_b200.pipeline import ReusePath
+    dp = hp.dev_pool(ab, pool)
+    model = hp.model_of(ab, w, n_layers=nl)
+    cap = ctx_cap or w.k * w.len_hi
+    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, cap, layers_per_call)
+    chunk = lambda x: [x[:, lb:le].contiguous().cuda() for lb, le in path.chunks]
+    out, H, fo = path.run(qs["q_emb"].cuda(), chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]),
+                          qs["logits"].cuda(), tau)
+    torch.cuda.synchronize()
+    assert path.status.item() == 0
+    return path, torch.cat(out, dim=1)
+
+
+def _to_bf16_inputs(w, pool, qs):
+    for key in ("k", "v"):
+        pool[key] = pool[key].to(torch.bfloat16)
+    for key in ("q", "kq", "vq"):
+        qs[key] = qs[key].to(torch.bfloat16)
+    return w.scaled(dtype="bf16")
+
+
+def _check(w, nl, layers_per_call=None, tau=None):
+    pool, qs = wl.make_pool(w, n_layers=nl), wl.make_queries(w, n_layers=nl)
+    if w.dtype == "fp32":     # the attention kernel is bf16: both sides get the same rounded inputs
+        w = _to_bf16_inputs(w, pool, qs)
+    H_want = orc.entropy(hp.f64(qs["logits"]))
+    tau = float(np.median(H_want)) + 1e-2 if tau is None else tau
+    sel, off, out_want, H_want, fo_want = oracle_path(w, pool, qs, nl, tau)
+    path, out = run_gpu_path(w, pool, qs, nl, tau, layers_per_call)
+    assert np.array_equal(path.sel_idx.cpu().numpy(), sel)
+    assert np.array_equal(path.ctx_off.cpu().numpy(), off)
+    err = np.abs(out.cpu().double().numpy() - out_want)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+    assert np.all(np.abs(path.H.cpu().numpy() - H_want) <= 1e-4 * np.abs(H_want))
+    assert np.array_equal(path.first_ok.cpu().numpy(), fo_want)
+
+
+def test_cfg1_whole_path():
+    _check(wl.CONFIGS["cfg1"], 1)
+
+
+def test_8b_shape_nested_probes_two_layer_chunks():
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=96, n_layers=3, batch=2, k=24, probes=(3, 6, 12, 24), t_q=48,
+                                  vocab=4000, seed=31)
+    _check(w, 3, layers_per_call=2)
