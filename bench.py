@@ -1,0 +1,448 @@
+#!/usr/bin/env python
+"""Benchmark of the AdapShot KV-reuse hot path on B200.
+
+One "step" = one pass of the whole path (select -> plan -> gather + RoPE re-encode ->
+probe attention -> entropy, all layers) over one batch of seeded synthetic queries.
+Metric: reused-context tokens/s = sum over queries of the assembled context length
+of the longest probe, per second of the whole step.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+N > 1 (launched by torch.distributed.run) runs independent replicas: the path has
+no exchange step, so ranks share nothing but the start/stop barrier ("weak" scaling).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_03644_b200 import workloads as wl
+
+METRIC = "reused-context tokens/s (select+re-encode+query attn)"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 512 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self._thr, self.nv = None, threading.Event(), None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def resolve_workload(name: str, probes_override=None) -> wl.Workload:
+    w = wl.CONFIGS[name]
+    if w.k == 0:      # cfg4: k = longest similarity-ordered prefix within the token limit; fixed at set-up
+        raise SystemExit("cfg4 is a parity configuration; bench workloads: cfg1 cfg2 cfg3 cfg5")
+    return w
+
+
+def algorithmic_counts(w: wl.Workload, ctx_off: np.ndarray, n_layers: int):
+    """Algorithmic bytes / flops of one step from the plan (per the design doc's per-unit figures)."""
+    L = ctx_off[:, -1].astype(np.float64)                         # longest probe per query
+    Lj = np.stack([ctx_off[:, n] for n in w.probes], axis=1).astype(np.float64)
+    bpt = w.bytes_per_token_layer
+    gather_bytes = float(L.sum()) * bpt * 2 * n_layers            # read + write, K and V
+    attn_flops = float((4.0 * w.t_q * (Lj + (w.t_q + 1) / 2.0) * w.n_q_heads * w.head_dim).sum()) * n_layers
+    attn_kv_bytes = float(L.sum()) * bpt * n_layers               # K/V of the longest probe read once
+    R = w.batch * len(w.probes)
+    entropy_bytes = float(R) * w.vocab * (4 if w.logits_dtype == "fp32" else 2)
+    select_bytes = float(wl.shot_lengths(w).size) * w.emb_dim * 4
+    return {"ctx_tokens": float(L.sum()), "gather_bytes": gather_bytes, "attn_flops": attn_flops,
+            "attn_kv_bytes": attn_kv_bytes, "entropy_bytes": entropy_bytes, "select_bytes": select_bytes}
+
+
+# ------------------------------------------------------------------ CPU oracle legs
+def oracle_sample_seconds(w: wl.Workload, pool, qs, row_stride: int):
+    """Times the oracle, as it stands, on a bounded sample of the workload: select,
+    offsets, assemble and entropy in full for query 0 / layer 0, attention on every
+    `row_stride`-th (probe, head, token) row; returns (seconds scaled to one full step,
+    description, measured seconds)."""
+    from oracle import adapshot_oracle as orc
+    f64 = wl.to_f64
+    t0 = time.perf_counter()
+    sel, _ = orc.select_topk(f64(qs["q_emb"]), f64(pool["emb"]), w.k)
+    off = orc.plan_offsets(sel, pool["shot_off"])
+    t_select = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kc, vc, _ = orc.assemble_kv(f64(pool["k"][:1]), f64(pool["v"][:1]), pool["shot_off"], sel[0], w.rope_base)
+    t_assemble = time.perf_counter() - t0
+    q, kq, vq = f64(qs["q"][0, 0]), f64(qs["kq"][0, 0]), f64(qs["vq"][0, 0])
+    rows = [(j, h, t) for j in range(len(w.probes)) for h in range(w.n_q_heads) for t in range(w.t_q)]
+    sample = rows[::row_stride]
+    t0 = time.perf_counter()
+    for j, h, t in sample:
+        orc.attn_row(q[j, t, h], kq[j], vq[j], kc[0], vc[0], int(off[0, w.probes[j]]), t, h // w.group, w.rope_base)
+    t_attn = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.entropy(f64(qs["logits"]))
+    t_entropy = time.perf_counter() - t0
+    units = w.batch * w.n_layers                                   # (query, layer) units are independent
+    full = t_select + t_entropy + units * (t_assemble + t_attn * len(rows) / len(sample))
+    measured = t_select + t_assemble + t_attn + t_entropy
+    desc = (f"select+entropy full; assemble and attention for query 0, layer 0 with every {row_stride}th of "
+            f"{len(rows)} attention rows; scaled by rows and by {units} (query, layer) units")
+    return full, desc, measured, float(off[:, -1].sum())
+
+
+def cpu_threads() -> int:
+    try:
+        import threadpoolctl
+        info = threadpoolctl.threadpool_info()
+        return max([i.get("num_threads", 1) for i in info] + [1])
+    except Exception:
+        return 1
+
+
+def host_inputs(w: wl.Workload, n_pool_layers: int = 1):
+    """CPU copies of a one-layer slice of the workload for the oracle legs."""
+    ws = w.scaled(batch=1)
+    pool = wl.make_pool(ws, "cpu", n_layers=n_pool_layers)
+    qs = wl.make_queries(ws, "cpu", n_layers=1)
+    return pool, qs
+
+
+def run_reference(args, w: wl.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    pool, qs = host_inputs(w)
+    n_rows = len(w.probes) * w.n_q_heads * w.t_q
+    stride = max(1, n_rows // 96)
+    for _ in range(args.warmup):
+        oracle_sample_seconds(w, pool, qs, stride * 8)
+    vals, desc, meas, ctx_tokens = [], "", 0.0, 0.0
+    for _ in range(args.steps):
+        full, desc, m, ctx1 = oracle_sample_seconds(w, pool, qs, stride)
+        vals.append(full)
+        meas += m
+        ctx_tokens = ctx1 * w.batch
+    sec = float(np.mean(vals))
+    value = ctx_tokens / sec
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "note": "oracle timed on host cores; each step is a bounded sample "
+                       "scaled to the full step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------- GPU arm
+def run_ours(args, w: wl.Workload):
+    from paper_2605_03644_b200 import binding as ab
+    from paper_2605_03644_b200.pipeline import ReusePath
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    dev = torch.device("cuda", local)
+
+    # ---- resident inputs (every rank: same pool, its own queries)
+    n_pool_layers = min(w.n_layers, args.pool_layers) if args.pool_layers else w.n_layers
+    pool = wl.make_pool(w, dev, n_layers=n_pool_layers)
+    wq = w.scaled(seed=w.seed + 100 * rank) if rank else w
+    lpc = args.layers_per_call or w.n_layers
+    so = torch.from_numpy(pool["shot_off"]).to(dev)
+    k_pool, v_pool = pool["k"], pool["v"]
+    if n_pool_layers < w.n_layers:
+        raise SystemExit("layer aliasing is not implemented; the pool must hold every layer")
+    dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
+    model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
+    ctx_cap = args.ctx_cap or w.k * w.len_hi
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc,
+                     attn_flags=args.attn_tiles_per_chunk)
+    qs = wl.make_queries(wq, dev)
+    chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
+    q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
+    del qs
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    launches_per_step = 2 + (1 if w.n_shots > 8192 else 0) + len(path.chunks) * (2 + 3) + 2
+
+    def step():
+        path.run(q_emb, qc, kqc, vqc, logits, args.tau)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- tighten the capacity to the planned context (set-up, not timed)
+    step()
+    torch.cuda.synchronize()
+    if path.status.item() != 0:
+        raise SystemExit(f"device status {path.status.item()}: {ab.adapshot_strerror(path.status.item())}")
+    ctx_off = path.ctx_off.cpu().numpy()
+    counts = algorithmic_counts(w, ctx_off, w.n_layers)
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+
+    # ---- timed region: K steps, CUDA events around every step, L2 flushed between steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    with ClockSampler(local) as clocks:
+        barrier()
+        for a, b in ev:
+            flush.zero_()
+            a.record()
+            step()
+            b.record()
+        barrier()
+    step_ms = np.array([a.elapsed_time(b) for a, b in ev])
+    total_ms = float(step_ms.sum())
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        tok = torch.tensor([counts["ctx_tokens"]], device=dev, dtype=torch.float64)
+        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
+        job_tokens = float(tok.item())
+    else:
+        job_tokens = counts["ctx_tokens"]
+    ms_per_step = total_ms / args.steps
+    value = job_tokens / (ms_per_step * 1e-3)
+    if path.status.item() != 0:
+        raise SystemExit(f"device status {path.status.item()} after the timed region")
+
+    # ---- per-call device times (second pass, same conditions) for the roofline object
+    names = ["select", "assemble", "attn", "entropy"]
+    acc = {n: 0.0 for n in names}
+    n_prof = min(args.steps, 50)
+    for _ in range(n_prof):
+        flush.zero_()
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(2 + 2 * len(path.chunks) + 1)]
+        marks[0].record()
+        path.select(q_emb)
+        marks[1].record()
+        mi = 1
+        for i, (lb, le) in enumerate(path.chunks):
+            path.assemble(lb, le)
+            marks[mi + 1].record()
+            path.attend(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
+            marks[mi + 2].record()
+            mi += 2
+        path.entropy(logits, args.tau)
+        marks[mi + 1].record()
+        torch.cuda.synchronize()
+        acc["select"] += marks[0].elapsed_time(marks[1])
+        mi = 1
+        for _c in path.chunks:
+            acc["assemble"] += marks[mi].elapsed_time(marks[mi + 1])
+            acc["attn"] += marks[mi + 1].elapsed_time(marks[mi + 2])
+            mi += 2
+        acc["entropy"] += marks[mi].elapsed_time(marks[mi + 1])
+    per_call_ms = {n: acc[n] / n_prof for n in names}
+
+    attn_s = per_call_ms["attn"] * 1e-3
+    gather_s = per_call_ms["assemble"] * 1e-3
+    attn_tflops = counts["attn_flops"] / attn_s / 1e12
+    attn_kv_gbs = counts["attn_kv_bytes"] / attn_s / 1e9
+    tensor_bound = counts["attn_flops"] / (peaks["bf16_tflops"] * 1e12) >= \
+        counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    roofline = {
+        "kernel": "attn_main (per adapshot_query_attn call: prep + main + combine)",
+        "bound": "tensor" if tensor_bound else "hbm",
+        "achieved": attn_tflops if tensor_bound else attn_kv_gbs,
+        "peak": peaks["bf16_tflops"] if tensor_bound else peaks["hbm_gbs"],
+        "unit": "TFLOP/s" if tensor_bound else "GB/s",
+        "frac": (attn_tflops / peaks["bf16_tflops"]) if tensor_bound else (attn_kv_gbs / peaks["hbm_gbs"]),
+        "frac_of_sustained_peak": attn_tflops / peaks["bf16_tflops_sustained"] if tensor_bound else None,
+        "peak_source": f"of {peaks['source']}",
+        "traffic": None,
+        "ms_per_step": per_call_ms["attn"],
+        "gather": {"bound": "hbm", "achieved": counts["gather_bytes"] / gather_s / 1e9, "peak": peaks["hbm_gbs"],
+                   "unit": "GB/s", "frac": counts["gather_bytes"] / gather_s / 1e9 / peaks["hbm_gbs"],
+                   "ms_per_step": per_call_ms["assemble"], "traffic": None},
+        "select": {"bound": "hbm", "achieved": counts["select_bytes"] / (per_call_ms["select"] * 1e-3) / 1e9,
+                   "unit": "GB/s", "ms_per_step": per_call_ms["select"]},
+        "entropy": {"bound": "hbm", "achieved": counts["entropy_bytes"] / (per_call_ms["entropy"] * 1e-3) / 1e9,
+                    "unit": "GB/s", "ms_per_step": per_call_ms["entropy"]},
+    }
+
+    # ---- end to end: pinned host inputs in, results out, inside the timed region
+    host = {"q_emb": q_emb.cpu().pin_memory(), "logits": logits.cpu().pin_memory(),
+            "q": [x.cpu().pin_memory() for x in qc], "kq": [x.cpu().pin_memory() for x in kqc],
+            "vq": [x.cpu().pin_memory() for x in vqc]}
+    out_host = [torch.empty_like(x, device="cpu").pin_memory() for x in path.out]
+    H_host = torch.empty_like(path.H, device="cpu").pin_memory()
+    fo_host = torch.empty_like(path.first_ok, device="cpu").pin_memory()
+    sel_host = torch.empty_like(path.sel_idx, device="cpu").pin_memory()
+    nbytes = lambda t: t.numel() * t.element_size()
+    h2d = nbytes(host["q_emb"]) + nbytes(host["logits"]) + sum(nbytes(x) for k in ("q", "kq", "vq") for x in host[k])
+    d2h = sum(nbytes(x) for x in out_host) + nbytes(H_host) + nbytes(fo_host) + nbytes(sel_host)
+
+    def e2e_step():
+        q_emb.copy_(host["q_emb"], non_blocking=True)
+        logits.copy_(host["logits"], non_blocking=True)
+        for i in range(len(path.chunks)):
+            qc[i].copy_(host["q"][i], non_blocking=True)
+            kqc[i].copy_(host["kq"][i], non_blocking=True)
+            vqc[i].copy_(host["vq"][i], non_blocking=True)
+        step()
+        for i in range(len(path.chunks)):
+            out_host[i].copy_(path.out[i], non_blocking=True)
+        H_host.copy_(path.H, non_blocking=True)
+        fo_host.copy_(path.first_ok, non_blocking=True)
+        sel_host.copy_(path.sel_idx, non_blocking=True)
+
+    n_e2e = max(3, min(args.steps, 50))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_e2e)]
+    for a, b in ev2:
+        flush.zero_()
+        a.record()
+        e2e_step()
+        b.record()
+    barrier()
+    e2e_ms = float(np.sum([a.elapsed_time(b) for a, b in ev2]))
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = job_tokens / (e2e_ms / n_e2e * 1e-3)
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        hpool, hqs = host_inputs(w)
+        n_rows = len(w.probes) * w.n_q_heads * w.t_q
+        full, desc, meas, ctx1 = oracle_sample_seconds(w, hpool, hqs, max(1, n_rows // 256))
+        cpu_baseline = {"value": ctx1 * w.batch / full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                        "sample": desc, "measured_seconds": meas}
+
+    if rank == 0:
+        clk = clocks.summary()
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
+                       "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool["n_shots"]),
+                       "pool_tokens": int(pool["pool_tokens"]), "ctx_tokens_per_step": counts["ctx_tokens"],
+                       "ctx_cap": ctx_cap, "layers_per_call": lpc, "l2": "flushed between steps (512 MiB write)",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clk,
+            "per_call_ms": per_call_ms,
+            "step_ms_min_med_max": [float(step_ms.min()), float(np.median(step_ms)), float(step_ms.max())],
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--layers-per-call", type=int, default=0)
+    ap.add_argument("--pool-layers", type=int, default=0)
+    ap.add_argument("--ctx-cap", type=int, default=0)
+    ap.add_argument("--attn-tiles-per-chunk", type=int, default=0)
+    ap.add_argument("--tau", type=float, default=0.65)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = resolve_workload(args.workload)
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, w)
+        return
+    small = w.n_layers == 1
+    args.steps = (1000 if small else 10) if args.steps is None else args.steps
+    args.warmup = (20 if small else 3) if args.warmup is None else max(3, args.warmup)
+    run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
