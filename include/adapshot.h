@@ -160,6 +160,30 @@ ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, 
                      float* H, float tau, int32_t rows_per_group, int32_t* first_ok,
                      void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
+/* ---- adapshot_entropy for callers that cannot provide or allocate scratch.
+ * (No counterpart in the paper: this is a packaging variant of the call above.)
+ * Meant for callers that must not call cudaMalloc, or hand out workspace, at the
+ * point where they need the probe entropy: code living inside a serving process
+ * whose device memory is fully owned by a pool allocator, plugins loaded into a
+ * host that forbids allocation after start-up, and paths where an allocation's
+ * implicit device synchronisation is not acceptable.  Same arguments, results
+ * and error codes as adapshot_entropy, minus `ws`: the per-split states live in
+ * a fixed 192 KiB device array inside the library (one per GPU that loads it,
+ * held until the process exits).
+ *  - Limit: R * splits <= 16384 states, where splits = min(ceil(296 / R),
+ *    ceil(V / 4096)); larger requests return ADAPSHOT_ECAPACITY and launch
+ *    nothing.  (Examples within the limit: 8 rows x 128256; 224 rows x 128256.)
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current); make that first call outside any stream capture.
+ *  - The call allocates and frees nothing, on the host or the device.
+ *  - All calls share the one array, and it keeps whatever the last call left in
+ *    it; every state a call reads is first written by that call, so stale
+ *    contents are harmless, but two calls whose kernels overlap on the GPU
+ *    (different streams, or different threads) race on it: serialise them.     */
+ADAPSHOT_API int adapshot_entropy_static(const void* logits, int32_t dtype, int32_t R, int32_t V,
+                            int64_t row_stride, float* H, float tau, int32_t rows_per_group,
+                            int32_t* first_ok, int32_t* status, void* stream);
+
 ADAPSHOT_API const char* adapshot_strerror(int code);
 ADAPSHOT_API int adapshot_version(void);
 

@@ -26,7 +26,7 @@ F32, BF16 = 0, 1
 EXPORTS = [
     "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
-    "adapshot_entropy_workspace_bytes", "adapshot_entropy",
+    "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_static",
     "adapshot_strerror", "adapshot_version",
 ]
 
@@ -58,6 +58,8 @@ _assemble = _sig("adapshot_assemble_kv", C.c_int,
 _entropy_ws = _sig("adapshot_entropy_workspace_bytes", _sz, [_i32, _i32])
 _entropy = _sig("adapshot_entropy", C.c_int,
                 [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _sz, _vp, _vp])
+_entropy_static = _sig("adapshot_entropy_static", C.c_int,
+                       [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _vp])
 _strerror = _sig("adapshot_strerror", C.c_char_p, [C.c_int])
 _version = _sig("adapshot_version", C.c_int, [])
 _attn_ws = _sig("adapshot_attn_workspace_bytes", _sz, [C.POINTER(ModelT), _i32, _i32, _i32, _i32, _i64])
@@ -167,3 +169,17 @@ def adapshot_entropy(logits: torch.Tensor, H: torch.Tensor, tau: float, rows_per
         raise ValueError("logit rows must be contiguous")
     _check(_entropy(logits.data_ptr(), dt, R, V, logits.stride(0), _ptr(H), tau, rows_per_group,
                     _ptr(first_ok), _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_entropy_static(logits: torch.Tensor, H: torch.Tensor, tau: float, rows_per_group: int,
+                            first_ok: Optional[torch.Tensor], status: torch.Tensor):
+    """adapshot_entropy for callers that may not allocate or pass scratch memory (for
+    instance code inside a server whose allocator owns all device memory): the scratch
+    is a fixed array inside the library.  Raises AdapshotError(ECAPACITY) beyond its
+    size.  Calls share that array, so do not let two of them overlap on the GPU."""
+    R, V = logits.shape
+    dt = F32 if logits.dtype == torch.float32 else BF16
+    if logits.stride(1) != 1:
+        raise ValueError("logit rows must be contiguous")
+    _check(_entropy_static(logits.data_ptr(), dt, R, V, logits.stride(0), _ptr(H), tau, rows_per_group,
+                           _ptr(first_ok), _ptr(status), _stream()))

@@ -194,3 +194,74 @@ extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, in
       partial, n_split, R, rows_per_group, tau, H, first_ok);
   return ads_launch_status();
 }
+
+
+// --------------------------------------------------------------------------
+// Entropy without any caller-provided or allocated scratch.
+//
+// Some callers may not allocate device memory at all: code running inside a
+// memory-pool-managed serving process whose allocator must not be bypassed, a
+// plugin loaded into a host that forbids cudaMalloc after start-up, or a
+// latency-critical path where an allocation could synchronise the device.  For
+// them the per-split states live in the fixed array below, which every GPU that
+// loads this library keeps until the process exits (192 KiB per device).
+constexpr int kStaticEntStates = 16384;   // most (row, split) states one call may need
+static __device__ __align__(256) float g_entropy_static_scratch[kStaticEntStates * 3];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+// In host code the array's name is only a handle for the runtime; the device
+// address has to be asked for, once per device, with that device current.
+int static_scratch_for_current_device(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ADAPSHOT_ECUDA;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_entropy_static_scratch) != cudaSuccess ||
+        ptr == nullptr)
+      return ADAPSHOT_ECUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return ADAPSHOT_OK;
+}
+}  // namespace
+
+extern "C" int adapshot_entropy_static(const void* logits, int32_t dtype, int32_t R, int32_t V,
+                                       int64_t row_stride, float* H, float tau, int32_t rows_per_group,
+                                       int32_t* first_ok, int32_t* status, void* stream) {
+  (void)status;
+  if (logits == nullptr || H == nullptr) return ADAPSHOT_EINVAL;
+  if (R <= 0 || V <= 0 || row_stride < V) return ADAPSHOT_EINVAL;
+  if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
+  if (rows_per_group <= 0) rows_per_group = 1;
+  if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
+  if (!ads_aligned16(logits) || (row_stride * es) % 16 != 0) return ADAPSHOT_EALIGN;
+  const int n_split = ent_splits(R, V);
+  if ((long long)R * n_split > kStaticEntStates) return ADAPSHOT_ECAPACITY;   // beyond the fixed array
+
+  float* partial = nullptr;
+  const int rc = static_scratch_for_current_device(&partial);
+  if (rc != ADAPSHOT_OK) return rc;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int vec = 16 / (int)es;
+  int slice = (V + n_split - 1) / n_split;
+  slice = (slice + vec - 1) / vec * vec;
+  dim3 grid(n_split, R);
+  // every (row, split) state this call reads is written by the first kernel, so
+  // nothing in the shared array has to start at zero
+  if (dtype == ADAPSHOT_F32)
+    entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(
+        static_cast<const float*>(logits), V, row_stride, slice, partial);
+  else
+    entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, partial);
+  if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  entropy_finish_kernel<<<R / rows_per_group, 256, rows_per_group * sizeof(float), st>>>(
+      partial, n_split, R, rows_per_group, tau, H, first_ok);
+  return ads_launch_status();
+}
