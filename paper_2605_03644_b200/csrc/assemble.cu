@@ -123,11 +123,14 @@ gather_rope_kernel(const GatherArgs a) {
   const long long layer_stride_pool = a.pool_tokens * row_vecs;   // in uint4
   const long long layer_stride_ctx = a.ctx_cap * row_vecs;
 
-  // theta of the EPV rotary pairs this lane owns (its vector column is fixed)
+  // theta_i once per CTA (fp64 pow is slow), then the EPV values of this lane's column
+  __shared__ double theta_sh[D / 2];
+  if (threadIdx.x < D / 2) theta_sh[threadIdx.x] = pow(a.rope_base, -2.0 * (double)threadIdx.x / (double)D);
+  __syncthreads();
   const int jcol = lane % HALF_V;
   double theta[EPV];
 #pragma unroll
-  for (int e = 0; e < EPV; ++e) theta[e] = pow(a.rope_base, -2.0 * (double)(jcol * EPV + e) / (double)D);
+  for (int e = 0; e < EPV; ++e) theta[e] = theta_sh[jcol * EPV + e];
 
   const uint4* kp = static_cast<const uint4*>(a.k_pool);
   const uint4* vp = static_cast<const uint4*>(a.v_pool);
@@ -168,7 +171,11 @@ gather_rope_kernel(const GatherArgs a) {
 
     float sn[EPV], cs[EPV];
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) rope_sincos(delta, theta[e], &sn[e], &cs[e]);
+    for (int e = 0; e < EPV; ++e) {
+      // bf16 storage rounds at 2^-9: the hardware sin/cos of the reduced angle is ample there
+      if constexpr (sizeof(T) == 2) rope_sincos_fast(delta, theta[e], &sn[e], &cs[e]);
+      else rope_sincos(delta, theta[e], &sn[e], &cs[e]);
+    }
 
     for (int l = 0; l < a.n_layers_call; ++l) {
       const long long src = (long long)(a.layer_begin + l) * layer_stride_pool + src_tok * row_vecs;

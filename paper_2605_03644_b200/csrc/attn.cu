@@ -65,6 +65,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint4 bf16x8_pack(const float* x) {
   return make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]),
                     pack_bf16x2(x[6], x[7]));
@@ -76,6 +81,9 @@ template <int D>
 __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   constexpr int VPH = D / 8, HALF_V = VPH / 2;
   const int lane = threadIdx.x & 31;
+  __shared__ double theta_sh[D / 2];   // theta_i once per CTA: fp64 pow is slow
+  if (threadIdx.x < D / 2) theta_sh[threadIdx.x] = pow(p.rope_base, -2.0 * (double)threadIdx.x / (double)D);
+  __syncthreads();
   const long long tok = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long n_tok = (long long)p.B * p.nl * p.P * p.Tq;
   if (tok >= n_tok) return;
@@ -91,8 +99,7 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   float sn[8], cs[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    const double theta = pow(p.rope_base, -2.0 * (double)(jcol * 8 + e) / (double)D);
-    rope_sincos(pos, theta, &sn[e], &cs[e]);
+    rope_sincos(pos, theta_sh[jcol * 8 + e], &sn[e], &cs[e]);
   }
   const uint4* qsrc = reinterpret_cast<const uint4*>(p.q) + tok * p.Hq * VPH;
   const uint4* ksrc = reinterpret_cast<const uint4*>(p.kq) + tok * p.Hkv * VPH;
@@ -331,7 +338,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       tc_fence_before();
       mbar_arrive(bar(kBarSEmpty + sb));
 
-      // mask: context keys at or beyond L_j; own keys after the row's token (causal)
+      // mask: context keys at or beyond L_j; own keys after the row's token (causal).
+      // Only the last context tile and the own-token tiles can hide anything.
       const bool own = i >= n_ctx;
       int limit = kTileN;                          // columns < limit are visible
       if (!own) {
@@ -342,14 +350,17 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int last_visible = min(t_row, p.Tq - 1);
         limit = last_visible - first + 1;          // may be <= 0: the whole tile is hidden
       }
-      float tile_max = -INFINITY;
+      if (__any_sync(0xffffffffu, limit < kTileN)) {
 #pragma unroll
-      for (int cidx = 0; cidx < kTileN; ++cidx) {
-        float v = s[cidx] * p.scale_log2;
-        v = cidx < limit ? v : -INFINITY;
-        s[cidx] = v;
-        tile_max = fmaxf(tile_max, v);
+        for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
       }
+      float mx[4] = {s[0], s[1], s[2], s[3]};
+#pragma unroll
+      for (int cidx = 4; cidx < kTileN; cidx += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], s[cidx + u]);
+      }
+      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
       float alpha = 1.f;
       const bool need = tile_max > m_used + kRescaleThreshold;
       if (need) {
@@ -373,19 +384,22 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           }
         }
       }
-      // P = 2^(s - m): row sum in fp32, bf16 tile into shared memory (K-major, swizzled)
+      // P = 2^(s * scale - m): row sum in fp32, bf16 tile into shared memory (K-major, swizzled)
       unsigned char* p_tile = base_ptr + AttnSmem::off_p<D>();
+      const float neg_m = -m_used;
+      float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ch = 0; ch < kTileN / 8; ++ch) {
         float e8[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          e8[e] = exp2f(s[ch * 8 + e] - m_used);
-          l_sum += e8[e];
+          e8[e] = ex2_approx(fmaf(s[ch * 8 + e], p.scale_log2, neg_m));
+          part[e & 3] += e8[e];
         }
         const uint32_t off = (ch / 8) * 16384u + r * 128u + (((ch % 8) ^ (r & 7)) << 4);
         *reinterpret_cast<uint4*>(p_tile + off) = bf16x8_pack(e8);
       }
+      l_sum += (part[0] + part[1]) + (part[2] + part[3]);
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar(kBarPFull));

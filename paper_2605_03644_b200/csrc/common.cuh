@@ -46,7 +46,7 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // Angle p * theta_i formed in fp64 and reduced to [-pi, pi] before the fp32
 // sincos, so that the result keeps fp32 accuracy at positions of 64K and more.
-__device__ __forceinline__ void rope_sincos(double delta, double theta, float* s, float* c) {
+__device__ __forceinline__ float rope_reduced_angle(double delta, double theta) {
   const double kInv2Pi = 0.15915494309189533577;
   const double k2PiHi = 6.283185307179586232;
   const double k2PiLo = 2.449293598294706354e-16;
@@ -54,5 +54,14 @@ __device__ __forceinline__ void rope_sincos(double delta, double theta, float* s
   double n = rint(a * kInv2Pi);
   double r = fma(-n, k2PiHi, a);
   r = fma(-n, k2PiLo, r);
-  sincosf(static_cast<float>(r), s, c);
+  return static_cast<float>(r);
+}
+__device__ __forceinline__ void rope_sincos(double delta, double theta, float* s, float* c) {
+  sincosf(rope_reduced_angle(delta, theta), s, c);
+}
+// Hardware approximations (absolute error below 1e-6 on [-pi, pi]): for bf16 storage only.
+__device__ __forceinline__ void rope_sincos_fast(double delta, double theta, float* s, float* c) {
+  const float r = rope_reduced_angle(delta, theta);
+  *s = __sinf(r);
+  *c = __cosf(r);
 }
