@@ -24,7 +24,6 @@ using namespace sm100;
 constexpr int kMaxProbes = 16;
 constexpr int kTileM = 128;          // query rows per CTA (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
-constexpr int kStages = 2;           // K/V ring depth
 constexpr int kAttnThreads = 192;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by 2^8
@@ -131,85 +130,129 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   }
 }
 
+constexpr int kMaxPairs = 256;       // (probe, query) pairs one call may hold: B * P <= 256
+
+// Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
+// written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
+template <int D>
 struct AttnSmem {
-  // offsets (bytes) from the 1024-aligned base; every operand tile is made of
-  // [128 rows][128 bytes] sub-tiles written by TMA with the 128-byte swizzle
-  template <int D> __host__ __device__ static constexpr uint32_t sub_tiles() { return D / 64; }
-  template <int D> __host__ __device__ static constexpr uint32_t q_bytes() { return sub_tiles<D>() * 16384u; }
-  template <int D> __host__ __device__ static constexpr uint32_t kv_bytes() { return sub_tiles<D>() * 16384u; }
-  __host__ __device__ static constexpr uint32_t p_bytes() { return 2 * 16384u; }
-  template <int D> __host__ __device__ static constexpr uint32_t off_q() { return 0; }
-  template <int D> __host__ __device__ static constexpr uint32_t off_k(int s) { return q_bytes<D>() + s * kv_bytes<D>(); }
-  template <int D> __host__ __device__ static constexpr uint32_t off_v(int s) { return q_bytes<D>() + (kStages + s) * kv_bytes<D>(); }
-  template <int D> __host__ __device__ static constexpr uint32_t off_p() { return q_bytes<D>() + 2 * kStages * kv_bytes<D>(); }
-  template <int D> __host__ __device__ static constexpr uint32_t off_bar() { return off_p<D>() + p_bytes(); }
-  template <int D> __host__ __device__ static constexpr uint32_t total() { return off_bar<D>() + 256 + 1024; }
+  static constexpr int kKStages = D == 128 ? 2 : 3;
+  static constexpr int kVStages = 3;
+  static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
+  static constexpr uint32_t kOffQ = 0;                                    // 2 buffers
+  static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
+  static constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
+  static constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
+  static constexpr uint32_t kOffPairs = kOffBar + 256;
+  static constexpr uint32_t kTotal = kOffPairs + (kMaxPairs + 1) * 4 + 1024;   // + alignment slack
 };
 
-enum Bar { kBarQ = 0, kBarKFull = 1, kBarVFull = 3, kBarKEmpty = 5, kBarVEmpty = 7, kBarSFull = 9,
-           kBarSEmpty = 11, kBarPFull = 13, kBarPVDone = 14, kBarDrain = 15, kNumBars = 16 };
+// mbarrier slots (8 bytes each)
+enum Bar {
+  kBarQFull = 0, kBarQEmpty = 2, kBarKFull = 4, kBarKEmpty = 7, kBarVFull = 10, kBarVEmpty = 13,
+  kBarSFull = 16, kBarPFull = 18, kBarPVDone = 20, kBarOFull = 21, kBarOEmpty = 23, kBarDrain = 25,
+  kNumBars = 26
+};
 
+struct WorkItem {
+  int b, l, j, g, mt, c;
+  long long Lj;
+  int t_begin, n_ctx, n_own, n_tiles;
+  int outer_ctx, outer_own, outer_q;
+  long long item_out;
+};
+
+// idx-th non-empty piece of work.  prefix[pi] = first index of pair pi = jj * B + b,
+// jj = P-1-j (longest probes first); inside a pair: chunk, layer, kv head, M tile
+// (M tile fastest, so CTAs that share a K/V chunk run at the same time).
+__device__ __forceinline__ void decode_item(const AttnParams& p, const int* prefix, int n_pairs, int idx,
+                                            WorkItem& w) {
+  int lo = 0, hi = n_pairs;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= idx) lo = mid; else hi = mid;
+  }
+  int local = idx - prefix[lo];
+  w.j = p.P - 1 - lo / p.B;
+  w.b = lo % p.B;
+  w.mt = local % p.n_mt; local /= p.n_mt;
+  w.g = local % p.Hkv; local /= p.Hkv;
+  w.l = local % p.nl;
+  w.c = local / p.nl;
+  long long Lj = p.ctx_off[(long long)w.b * (p.k + 1) + p.nshots[w.j]];
+  Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
+  w.Lj = Lj;
+  const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
+  const int c_last = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk : 0;
+  w.t_begin = w.c * p.tiles_per_chunk;
+  w.n_ctx = max(0, min(n_tiles_ctx, w.t_begin + p.tiles_per_chunk) - w.t_begin);
+  w.n_own = 0;
+  if (w.c == c_last) {   // the last chunk also takes the probe's own tokens (causal part)
+    const int row_hi = min(p.Tq * p.G - 1, w.mt * kTileM + kTileM - 1);
+    w.n_own = (row_hi / p.G) / kTileN + 1;
+  }
+  w.n_tiles = w.n_ctx + w.n_own;
+  w.outer_ctx = w.b * p.nl + w.l;
+  w.outer_own = w.outer_ctx * p.P + w.j;
+  w.outer_q = w.outer_own * p.Hkv + w.g;
+  w.item_out = (((long long)w.outer_own * p.Hkv + w.g) * p.n_mt + w.mt) * p.n_chunks + w.c;
+}
+
+// Persistent kernel: one CTA per SM walks over the non-empty work items round-robin.
+// TMEM: S/P buffers at columns 0 and 128 (P, as packed bf16, overwrites the S tile it
+// was computed from), O accumulators at 256 and 384 (alternating per item so that the
+// read-out of one item overlaps the MMAs of the next).
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
                  const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
-  constexpr int SUB = D / 64;                      // 64-column sub-tiles per operand row
-  constexpr uint32_t kTileBytes = SUB * 16384u;
+  using SM = AttnSmem<D>;
+  constexpr int SUB = D / 64;
+  constexpr int KS = SM::kKStages, VS = SM::kVStages;
+  constexpr uint32_t kTileBytes = SM::kTileBytes;
   constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, 0);
   constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, 1);
   constexpr uint32_t kTmemS = 0, kTmemO = 256;
-
-  // ---- which piece of work is this CTA
-  int item = blockIdx.x;
-  const int mt = item % p.n_mt; item /= p.n_mt;
-  const int g = item % p.Hkv; item /= p.Hkv;
-  const int c = item % p.n_chunks; item /= p.n_chunks;
-  const int l = item % p.nl; item /= p.nl;
-  const int b = item % p.B; item /= p.B;
-  const int j = p.P - 1 - item;                    // longest probes are launched first
-
-  long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
-  if (Lj > p.ctx_cap) Lj = p.ctx_cap;
-  if (Lj < 0) Lj = 0;
-  const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
-  const int c_last = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk : 0;
-  if (c > c_last) return;                          // empty chunk: the combine step skips it too
-  const int t_begin = c * p.tiles_per_chunk;
-  const int t_end = min(n_tiles_ctx, t_begin + p.tiles_per_chunk);
-  const int n_ctx = max(0, t_end - t_begin);
-  const int M_total = p.Tq * p.G;
-  int n_own = 0;
-  if (c == c_last) {
-    const int row_hi = min(M_total - 1, mt * kTileM + kTileM - 1);
-    n_own = (row_hi / p.G) / kTileN + 1;           // own key tiles holding t' <= t of the last row
-  }
-  const int n_tiles = n_ctx + n_own;               // >= 1
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_raw + (base - raw_addr);
-  const uint32_t bar0 = base + AttnSmem::off_bar<D>();
+  const uint32_t bar0 = base + SM::kOffBar;
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + AttnSmem::off_bar<D>() + 8 * kNumBars);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + AttnSmem::off_bar<D>() + 8 * kNumBars + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + SM::kOffBar + 8 * kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + SM::kOffBar + 8 * kNumBars + 8);
+  int* prefix = reinterpret_cast<int*>(base_ptr + SM::kOffPairs);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_pairs = p.P * p.B;
 
+  // ---- how many non-empty items every (probe, query) pair has
+  const int per_chunk = p.nl * p.Hkv * p.n_mt;
+  for (int pi = threadIdx.x; pi < n_pairs; pi += kAttnThreads) {
+    const int j = p.P - 1 - pi / p.B, b = pi % p.B;
+    long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
+    Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
+    const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
+    const int n_valid = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk + 1 : 1;
+    prefix[pi + 1] = n_valid * per_chunk;
+  }
   if (threadIdx.x == 32) {
-    mbar_init(bar(kBarQ), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar(kBarKFull + s), 1);
-      mbar_init(bar(kBarVFull + s), 1);
-      mbar_init(bar(kBarKEmpty + s), 1);
-      mbar_init(bar(kBarVEmpty + s), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(kBarQFull + i), 1);
+      mbar_init(bar(kBarQEmpty + i), 1);
+      mbar_init(bar(kBarSFull + i), 1);
+      mbar_init(bar(kBarPFull + i), 128);
+      mbar_init(bar(kBarOFull + i), 1);
+      mbar_init(bar(kBarOEmpty + i), 128);
     }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(kBarSFull + s), 1);
-      mbar_init(bar(kBarSEmpty + s), 128);
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(bar(kBarKFull + i), 1);
+      mbar_init(bar(kBarKEmpty + i), 1);
+      mbar_init(bar(kBarVFull + i), 1);
+      mbar_init(bar(kBarVEmpty + i), 1);
     }
-    mbar_init(bar(kBarPFull), 128);
     mbar_init(bar(kBarPVDone), 1);
     mbar_init(bar(kBarDrain), 1);
     abort_flag[0] = 0;
@@ -222,95 +265,125 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) {
+    prefix[0] = 0;
+    for (int pi = 0; pi < n_pairs; ++pi) prefix[pi + 1] += prefix[pi];
+  }
+  __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-
-  const int outer_ctx = b * p.nl + l;
-  const int outer_own = (b * p.nl + l) * p.P + j;
-  const int outer_q = outer_own * p.Hkv + g;
+  const int total = prefix[n_pairs];
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kctx); tma_prefetch_desc(&tm_vctx);
-      mbar_arrive_expect_tx(bar(kBarQ), kTileBytes);
-#pragma unroll
-      for (int s = 0; s < SUB; ++s)
-        tma_load_3d(base + AttnSmem::off_q<D>() + s * 16384u, &tm_q, bar(kBarQ), s * 64, mt * kTileM, outer_q);
-      int issued_k = 0, issued_v = 0;
+      uint32_t tk = 0, tv = 0;
+      int n = 0;
       bool ok = true;
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        const int st = i % kStages;
-        ok = mbar_wait(bar(kBarKEmpty + st), ((i / kStages) & 1) ^ 1, abort_flag);
+      for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
+        WorkItem w;
+        decode_item(p, prefix, n_pairs, idx, w);
+        const int qb = n & 1;
+        ok = mbar_wait(bar(kBarQEmpty + qb), ((n >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
-        const bool own = i >= n_ctx;
-        const CUtensorMap* mk = own ? &tm_kown : &tm_kctx;
-        const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
-        const int row = own ? (i - n_ctx) * kTileN : (t_begin + i) * kTileN;
-        const int outer = own ? outer_own : outer_ctx;
-        mbar_arrive_expect_tx(bar(kBarKFull + st), kTileBytes);
+        mbar_arrive_expect_tx(bar(kBarQFull + qb), kTileBytes);
 #pragma unroll
         for (int s = 0; s < SUB; ++s)
-          tma_load_4d(base + AttnSmem::off_k<D>(st) + s * 16384u, mk, bar(kBarKFull + st), s * 64, g, row, outer);
-        issued_k = i + 1;
-        ok = mbar_wait(bar(kBarVEmpty + st), ((i / kStages) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(kBarVFull + st), kTileBytes);
+          tma_load_3d(base + SM::kOffQ + qb * kTileBytes + s * 16384u, &tm_q, bar(kBarQFull + qb), s * 64,
+                      w.mt * kTileM, w.outer_q);
+        for (int i = 0; i < w.n_tiles; ++i) {
+          const bool own = i >= w.n_ctx;
+          const CUtensorMap* mk = own ? &tm_kown : &tm_kctx;
+          const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
+          const int row = own ? (i - w.n_ctx) * kTileN : (w.t_begin + i) * kTileN;
+          const int outer = own ? w.outer_own : w.outer_ctx;
+          const int sk = tk % KS;
+          ok = mbar_wait(bar(kBarKEmpty + sk), ((tk / KS) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar(kBarKFull + sk), kTileBytes);
 #pragma unroll
-        for (int s = 0; s < SUB; ++s)
-          tma_load_4d(base + AttnSmem::off_v<D>(st) + s * 16384u, mv, bar(kBarVFull + st), s * 64, g, row, outer);
-        issued_v = i + 1;
+          for (int s = 0; s < SUB; ++s)
+            tma_load_4d(base + SM::kOffK + sk * kTileBytes + s * 16384u, mk, bar(kBarKFull + sk), s * 64, w.g, row,
+                        outer);
+          ++tk;
+          const int sv = tv % VS;
+          ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
+#pragma unroll
+          for (int s = 0; s < SUB; ++s)
+            tma_load_4d(base + SM::kOffV + sv * kTileBytes + s * 16384u, mv, bar(kBarVFull + sv), s * 64, w.g, row,
+                        outer);
+          ++tv;
+        }
       }
       if (!ok) {
         // gave up: let the copies already in flight land before the CTA retires
-        for (int i = max(0, issued_k - kStages); i < issued_k; ++i)
-          mbar_wait(bar(kBarKFull + i % kStages), (i / kStages) & 1, abort_flag + 1);
-        for (int i = max(0, issued_v - kStages); i < issued_v; ++i)
-          mbar_wait(bar(kBarVFull + i % kStages), (i / kStages) & 1, abort_flag + 1);
-        mbar_wait(bar(kBarQ), 0, abort_flag + 1);
+        for (uint32_t t = tk > (uint32_t)KS ? tk - KS : 0; t < tk; ++t)
+          mbar_wait(bar(kBarKFull + t % KS), (t / KS) & 1, abort_flag + 1);
+        for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
+          mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
+        for (int t = max(0, n - 1); t <= n; ++t)
+          mbar_wait(bar(kBarQFull + (t & 1)), (t >> 1) & 1, abort_flag + 1);
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      bool ok = mbar_wait(bar(kBarQ), 0, abort_flag);
-      auto issue_pv = [&](int i) -> bool {
-        const int st = i % kStages;
-        if (!mbar_wait(bar(kBarPFull), i & 1, abort_flag)) return false;
-        if (!mbar_wait(bar(kBarVFull + st), (i / kStages) & 1, abort_flag)) return false;
+      struct Pending { int sb, sv, vphase, pphase, ob, ophase, first, last; };
+      Pending prev{};
+      bool have_prev = false, ok = true;
+      auto issue_pv = [&](const Pending& t) -> bool {
+        if (t.first && !mbar_wait(bar(kBarOEmpty + t.ob), t.ophase ^ 1, abort_flag)) return false;
+        if (!mbar_wait(bar(kBarPFull + t.sb), t.pphase, abort_flag)) return false;
+        if (!mbar_wait(bar(kBarVFull + t.sv), t.vphase, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t p_base = base + AttnSmem::off_p<D>();
-        const uint32_t v_base = base + AttnSmem::off_v<D>(st);
+        const uint32_t v_base = base + SM::kOffV + t.sv * kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kTileN / 16; ++ks) {
-          const uint64_t a = smem_desc_sw128(p_base + (ks / 4) * 16384u + (ks % 4) * 32u, 16, 1024);
-          const uint64_t bd = smem_desc_sw128(v_base + ks * 2048u, 16384, 1024);
-          umma_ss(tmem_base + kTmemO, a, bd, kIdescPV, (i > 0 || ks > 0) ? 1u : 0u);
+          // A = P from TMEM: 16 bf16 keys of one k-step occupy 8 packed columns
+          umma_ts(tmem_base + kTmemO + t.ob * 128, tmem_base + kTmemS + t.sb * kTileN + ks * 8,
+                  smem_desc_sw128(v_base + ks * 2048u, 16384, 1024), kIdescPV, (!t.first || ks > 0) ? 1u : 0u);
         }
-        umma_commit(bar(kBarVEmpty + st));
+        umma_commit(bar(kBarVEmpty + t.sv));
         umma_commit(bar(kBarPVDone));
+        if (t.last) umma_commit(bar(kBarOFull + t.ob));
         return true;
       };
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        const int st = i % kStages, sb = i & 1;
-        ok = mbar_wait(bar(kBarKFull + st), (i / kStages) & 1, abort_flag) &&
-             mbar_wait(bar(kBarSEmpty + sb), ((i >> 1) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t q_base = base + AttnSmem::off_q<D>();
-        const uint32_t k_base = base + AttnSmem::off_k<D>(st);
+      uint32_t tk = 0, tv = 0, gt = 0;
+      int n = 0;
+      for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
+        WorkItem w;
+        decode_item(p, prefix, n_pairs, idx, w);
+        const int qb = n & 1;
+        ok = mbar_wait(bar(kBarQFull + qb), (n >> 1) & 1, abort_flag);
+        const uint32_t q_base = base + SM::kOffQ + qb * kTileBytes;
+        for (int i = 0; i < w.n_tiles && ok; ++i) {
+          const int sk = tk % KS, sb = gt & 1;
+          ok = mbar_wait(bar(kBarKFull + sk), (tk / KS) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_base = base + SM::kOffK + sk * kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t o = (ks / 4) * 16384u + (ks % 4) * 32u;
-          umma_ss(tmem_base + kTmemS + sb * kTileN, smem_desc_sw128(q_base + o, 16, 1024),
-                  smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t o = (ks / 4) * 16384u + (ks % 4) * 32u;
+            umma_ss(tmem_base + kTmemS + sb * kTileN, smem_desc_sw128(q_base + o, 16, 1024),
+                    smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(bar(kBarSFull + sb));
+          umma_commit(bar(kBarKEmpty + sk));
+          if (i == w.n_tiles - 1) umma_commit(bar(kBarQEmpty + qb));
+          ++tk;
+          if (have_prev) ok = issue_pv(prev);
+          prev.sb = sb; prev.sv = tv % VS; prev.vphase = (tv / VS) & 1; prev.pphase = (gt >> 1) & 1;
+          prev.ob = n & 1; prev.ophase = (n >> 1) & 1; prev.first = i == 0; prev.last = i == w.n_tiles - 1;
+          have_prev = true;
+          ++tv; ++gt;
         }
-        umma_commit(bar(kBarSFull + sb));
-        umma_commit(bar(kBarKEmpty + st));
-        if (i > 0) ok = issue_pv(i - 1);
       }
-      if (ok) ok = issue_pv(n_tiles - 1);
+      if (ok && have_prev) ok = issue_pv(prev);
       if (!ok) {
         umma_commit(bar(kBarDrain));
         mbar_wait(bar(kBarDrain), 0, abort_flag + 1);
@@ -322,103 +395,103 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int quarter = warp & 3;                  // TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;             // row of the M tile
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    const int row_global = mt * kTileM + r;
-    const int t_row = row_global / p.G;            // probe token of this row
-    float m_used = kNegSentinel, l_sum = 0.f;
+    uint32_t gt = 0;
+    int n = 0;
     bool ok = true;
-    for (int i = 0; i < n_tiles && ok; ++i) {
-      const int sb = i & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + sb), (i >> 1) & 1, abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      float s[kTileN];
-#pragma unroll
-      for (int q4 = 0; q4 < kTileN / 32; ++q4)
-        tmem_ld32(tmem_base + lane_addr + kTmemS + sb * kTileN + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-      tc_fence_before();
-      mbar_arrive(bar(kBarSEmpty + sb));
-
-      // mask: context keys at or beyond L_j; own keys after the row's token (causal).
-      // Only the last context tile and the own-token tiles can hide anything.
-      const bool own = i >= n_ctx;
-      int limit = kTileN;                          // columns < limit are visible
-      if (!own) {
-        const long long first = (long long)(t_begin + i) * kTileN;
-        if (first + kTileN > Lj) limit = (int)(Lj - first);
-      } else {
-        const int first = (i - n_ctx) * kTileN;
-        const int last_visible = min(t_row, p.Tq - 1);
-        limit = last_visible - first + 1;          // may be <= 0: the whole tile is hidden
-      }
-      if (__any_sync(0xffffffffu, limit < kTileN)) {
-#pragma unroll
-        for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
-      }
-      float mx[4] = {s[0], s[1], s[2], s[3]};
-#pragma unroll
-      for (int cidx = 4; cidx < kTileN; cidx += 4) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], s[cidx + u]);
-      }
-      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
-      float alpha = 1.f;
-      const bool need = tile_max > m_used + kRescaleThreshold;
-      if (need) {
-        alpha = exp2f(m_used - tile_max);
-        m_used = tile_max;
-        l_sum *= alpha;
-      }
-      if (i > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPVDone), (i - 1) & 1, abort_flag));   // P free, O stable
+    for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
+      WorkItem w;
+      decode_item(p, prefix, n_pairs, idx, w);
+      const int ob = n & 1;
+      const int t_row = (w.mt * kTileM + r) / p.G;   // probe token of this row
+      float m_used = kNegSentinel, l_sum = 0.f;
+      for (int i = 0; i < w.n_tiles; ++i, ++gt) {
+        const int sb = gt & 1;
+        const uint32_t s_addr = tmem_base + lane_addr + kTmemS + sb * kTileN;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + sb), (gt >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, need)) {
+        float s[kTileN];
 #pragma unroll
-          for (int q4 = 0; q4 < D / 32; ++q4) {
-            float o[32];
-            const uint32_t addr = tmem_base + lane_addr + kTmemO + q4 * 32;
-            tmem_ld32(addr, reinterpret_cast<uint32_t*>(o));
+        for (int q4 = 0; q4 < kTileN / 32; ++q4) tmem_ld32(s_addr + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+
+        // mask: context keys at or beyond L_j; own keys after the row's token (causal).
+        // Only the last context tile and the own-token tiles can hide anything.
+        int limit = kTileN;                          // columns < limit are visible
+        if (i < w.n_ctx) {
+          const long long first = (long long)(w.t_begin + i) * kTileN;
+          if (first + kTileN > w.Lj) limit = (int)(w.Lj - first);
+        } else {
+          limit = min(t_row, p.Tq - 1) - (i - w.n_ctx) * kTileN + 1;   // <= 0: the whole tile is hidden
+        }
+        if (__any_sync(0xffffffffu, limit < kTileN)) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] *= alpha;
-            tmem_st32(addr, reinterpret_cast<const uint32_t*>(o));
+          for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
+        }
+        float mx[4] = {s[0], s[1], s[2], s[3]};
+#pragma unroll
+        for (int cidx = 4; cidx < kTileN; cidx += 4) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], s[cidx + u]);
+        }
+        const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
+        float alpha = 1.f;
+        const bool need = tile_max > m_used + kRescaleThreshold;
+        if (need) {
+          alpha = exp2f(m_used - tile_max);
+          m_used = tile_max;
+          l_sum *= alpha;
+        }
+        // P = 2^(s * scale - m) as packed bf16 back into the S columns (two keys per column)
+        const float neg_m = -m_used;
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pk[kTileN / 2];
+#pragma unroll
+        for (int c2 = 0; c2 < kTileN / 2; ++c2) {
+          const float e0 = ex2_approx(fmaf(s[2 * c2], p.scale_log2, neg_m));
+          const float e1 = ex2_approx(fmaf(s[2 * c2 + 1], p.scale_log2, neg_m));
+          part[c2 & 1] += e0;
+          part[2 + (c2 & 1)] += e1;
+          pk[c2] = pack_bf16x2(e0, e1);
+        }
+        l_sum += (part[0] + part[1]) + (part[2] + part[3]);
+        tmem_st32(s_addr, pk);
+        tmem_st32(s_addr + 32, pk + 32);
+        if (i > 0) {
+          // O may only be rescaled between PV(i-1) and PV(i)
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPVDone), (gt - 1) & 1, abort_flag));
+          if (!ok) break;
+          if (__any_sync(0xffffffffu, need)) {
+            tc_fence_after();
+#pragma unroll
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+              float o[32];
+              const uint32_t addr = tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32;
+              tmem_ld32(addr, reinterpret_cast<uint32_t*>(o));
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] *= alpha;
+              tmem_st32(addr, reinterpret_cast<const uint32_t*>(o));
+            }
           }
         }
+        tc_fence_before();
+        mbar_arrive(bar(kBarPFull + sb));
       }
-      // P = 2^(s * scale - m): row sum in fp32, bf16 tile into shared memory (K-major, swizzled)
-      unsigned char* p_tile = base_ptr + AttnSmem::off_p<D>();
-      const float neg_m = -m_used;
-      float part[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int ch = 0; ch < kTileN / 8; ++ch) {
-        float e8[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          e8[e] = ex2_approx(fmaf(s[ch * 8 + e], p.scale_log2, neg_m));
-          part[e & 3] += e8[e];
-        }
-        const uint32_t off = (ch / 8) * 16384u + r * 128u + (((ch % 8) ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(p_tile + off) = bf16x8_pack(e8);
-      }
-      l_sum += (part[0] + part[1]) + (part[2] + part[3]);
-      fence_proxy_async_smem();
-      tc_fence_before();
-      mbar_arrive(bar(kBarPFull));
-    }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPVDone), (n_tiles - 1) & 1, abort_flag));
-    if (ok) {
+      if (!ok) break;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (n >> 1) & 1, abort_flag));
+      if (!ok) break;
       tc_fence_after();
-      const long long item_out =
-          ((((long long)outer_own * p.Hkv + g) * p.n_mt + mt) * p.n_chunks + c);
-      float* orow = p.o_part + (item_out * kTileM + r) * D;
+      float* orow = p.o_part + (w.item_out * kTileM + r) * D;
 #pragma unroll
       for (int q4 = 0; q4 < D / 32; ++q4) {
         float o[32];
-        tmem_ld32(tmem_base + lane_addr + kTmemO + q4 * 32, reinterpret_cast<uint32_t*>(o));
+        tmem_ld32(tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32, reinterpret_cast<uint32_t*>(o));
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
           *reinterpret_cast<float4*>(orow + q4 * 32 + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
       }
-      float* ml = p.ml_part + (item_out * kTileM + r) * 2;
+      tc_fence_before();
+      mbar_arrive(bar(kBarOEmpty + ob));
+      float* ml = p.ml_part + (w.item_out * kTileM + r) * 2;
       ml[0] = m_used;
       ml[1] = l_sum;
     }
@@ -618,13 +691,20 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
   for (int i = 0; i < kMaxProbes; ++i) ap.nshots[i] = pp.nshots[i];
-  const int smem = (int)AttnSmem::total<128>();    // same request for D = 64: one CTA per SM
+  const int smem = (int)AttnSmem<128>::kTotal;     // same request for D = 64: one CTA per SM
   static bool attr_done[2] = {false, false};
   if (!attr_done[D == 128]) {
     ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done[D == 128] = true;
   }
-  attn_main_kernel<D><<<(unsigned)pl.items, kAttnThreads, smem, st>>>(tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    ADS_CHECK_CUDA(cudaGetDevice(&dev));
+    ADS_CHECK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const unsigned grid = (unsigned)(pl.items < n_sm ? pl.items : n_sm);   // persistent: one CTA per SM
+  attn_main_kernel<D><<<grid, kAttnThreads, smem, st>>>(tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   // ---- merge
@@ -665,7 +745,7 @@ extern "C" int adapshot_query_attn(const adapshot_model_t* model, const void* k_
   if (model->dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
   if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
   if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
-  if (P < 1 || P > kMaxProbes) return ADAPSHOT_ESHAPE;
+  if (P < 1 || P > kMaxProbes || (long long)P * B > kMaxPairs) return ADAPSHOT_ESHAPE;
   for (int i = 0; i < P; ++i) {
     if (probe_nshots[i] < 1 || probe_nshots[i] > k) return ADAPSHOT_ESHAPE;
     if (i > 0 && probe_nshots[i] <= probe_nshots[i - 1]) return ADAPSHOT_ESHAPE;
