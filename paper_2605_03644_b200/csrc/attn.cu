@@ -411,8 +411,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!ok) break;
         tc_fence_after();
         float s[kTileN];
-#pragma unroll
-        for (int q4 = 0; q4 < kTileN / 32; ++q4) tmem_ld32(s_addr + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+        tmem_ld128(s_addr, reinterpret_cast<uint32_t*>(s));
 
         // mask: context keys at or beyond L_j; own keys after the row's token (causal).
         // Only the last context tile and the own-token tiles can hide anything.
@@ -427,11 +426,11 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
           for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
         }
-        float mx[4] = {s[0], s[1], s[2], s[3]};
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int cidx = 4; cidx < kTileN; cidx += 4) {
+        for (int cidx = 0; cidx < kTileN; cidx += 8) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], s[cidx + u]);
+          for (int u = 0; u < 4; ++u) mx[u] = fmax3(mx[u], s[cidx + 2 * u], s[cidx + 2 * u + 1]);
         }
         const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
         float alpha = 1.f;
@@ -441,36 +440,36 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           m_used = tile_max;
           l_sum *= alpha;
         }
-        // P = 2^(s * scale - m) as packed bf16 back into the S columns (two keys per column)
-        const float neg_m = -m_used;
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
+        // P = 2^(s * scale - m) as packed bf16 back into the S columns (two keys per column);
+        // scale-and-shift and the row sum run two columns per instruction (packed fp32)
+        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+        const float2 neg_m2 = make_float2(-m_used, -m_used);
+        float2 part[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
         uint32_t pk[kTileN / 2];
 #pragma unroll
         for (int c2 = 0; c2 < kTileN / 2; ++c2) {
-          const float e0 = ex2_approx(fmaf(s[2 * c2], p.scale_log2, neg_m));
-          const float e1 = ex2_approx(fmaf(s[2 * c2 + 1], p.scale_log2, neg_m));
-          part[c2 & 1] += e0;
-          part[2 + (c2 & 1)] += e1;
-          pk[c2] = pack_bf16x2(e0, e1);
+          const float2 x = __ffma2_rn(make_float2(s[2 * c2], s[2 * c2 + 1]), scale2, neg_m2);
+          const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+          part[c2 & 3] = __fadd2_rn(part[c2 & 3], e);
+          pk[c2] = pack_bf16x2(e.x, e.y);
         }
-        l_sum += (part[0] + part[1]) + (part[2] + part[3]);
-        tmem_st32(s_addr, pk);
-        tmem_st32(s_addr + 32, pk + 32);
-        if (i > 0) {
-          // O may only be rescaled between PV(i-1) and PV(i)
+        const float2 tot = __fadd2_rn(__fadd2_rn(part[0], part[1]), __fadd2_rn(part[2], part[3]));
+        l_sum += tot.x + tot.y;
+        tmem_st64(s_addr, pk);
+        if (i > 0 && __any_sync(0xffffffffu, need)) {
+          // O may only be rescaled between PV(i-1) and PV(i).  PV(i) cannot start before this
+          // thread has arrived on PFull below, so the barrier is never more than one phase ahead.
           ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPVDone), (gt - 1) & 1, abort_flag));
           if (!ok) break;
-          if (__any_sync(0xffffffffu, need)) {
-            tc_fence_after();
+          tc_fence_after();
 #pragma unroll
-            for (int q4 = 0; q4 < D / 32; ++q4) {
-              float o[32];
-              const uint32_t addr = tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32;
-              tmem_ld32(addr, reinterpret_cast<uint32_t*>(o));
+          for (int q4 = 0; q4 < D / 32; ++q4) {
+            float o[32];
+            const uint32_t addr = tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32;
+            tmem_ld32(addr, reinterpret_cast<uint32_t*>(o));
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] *= alpha;
-              tmem_st32(addr, reinterpret_cast<const uint32_t*>(o));
-            }
+            for (int e = 0; e < 32; ++e) o[e] *= alpha;
+            tmem_st32(addr, reinterpret_cast<const uint32_t*>(o));
           }
         }
         tc_fence_before();
