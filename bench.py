@@ -232,8 +232,7 @@ def run_ours(args, w: wl.Workload):
     dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
     ctx_cap = args.ctx_cap or w.k * w.len_hi
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc,
-                     attn_flags=args.attn_tiles_per_chunk)
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc)
     qs = wl.make_queries(wq, dev)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
@@ -428,7 +427,6 @@ def main():
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--pool-layers", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
-    ap.add_argument("--attn-tiles-per-chunk", type=int, default=0)
     ap.add_argument("--tau", type=float, default=0.65)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

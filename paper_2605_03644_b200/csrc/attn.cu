@@ -3,14 +3,21 @@
 // tokens; scores scaled by 1/sqrt(d) as in Eq. 5; rotary positions of Eq. 6).
 //
 // Three kernels:
-//   attn_prep     rotates Q and the probe's own K to their positions L_j + t and
-//                 packs Q rows of one KV head (GQA) into an M-major tile layout;
-//   attn_main     one CTA per (query, layer, probe, kv head, 128-row M tile, context
-//                 chunk): TMA stages K/V tiles, tcgen05 UMMA computes S = Q K^T and
-//                 O += P V with accumulators in TMEM, four warps run the online
-//                 softmax (one thread per row); un-normalised partial results go to
-//                 the workspace;
-//   attn_combine  log-sum-exp merge of the chunk partials, normalise, store bf16.
+//   attn_prep     rotates Q and the probe's own K to their positions L_j + t, packs the
+//                 Q rows of one KV head (GQA) into an M-major tile layout, and writes
+//                 the schedule (how many 128-key tiles every (probe, query) pair has
+//                 and how the tile sequence is cut into equal ranges);
+//   attn_main     persistent CTAs.  A CTA works on two 128-row M tiles of one KV head
+//                 at a time ("M pair"): TMA stages each K/V tile once for both, one
+//                 thread issues tcgen05 UMMAs (S = Q K^T, O += P V, accumulators in
+//                 TMEM, P kept in TMEM), two groups of four warps run the online
+//                 softmax of the two M tiles (one thread per row) and alternate on the
+//                 tensor pipe.  The global tile sequence is cut into equal ranges, one
+//                 per gang of CTAs (the CTAs of a gang take the M pairs of the same
+//                 K/V tiles, so the tiles are shared through L2).  A range that covers
+//                 a whole unit stores the final bf16 rows; a range that cuts a unit
+//                 stores un-normalised partials;
+//   attn_combine  log-sum-exp merge of the partials of the cut units.
 #include <cuda.h>
 #include <float.h>
 
@@ -22,23 +29,40 @@ namespace {
 using namespace sm100;
 
 constexpr int kMaxProbes = 16;
-constexpr int kTileM = 128;          // query rows per CTA (TMEM lanes)
+constexpr int kMaxPairs = 256;       // (probe, query) pairs one call may hold: B * P <= 256
+constexpr int kMaxCtas = 160;        // persistent grid: one CTA per SM, at most this many
+constexpr int kMaxGang = 8;          // CTAs that share one range of K/V tiles
+constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
-constexpr int kAttnThreads = 192;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax
+constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by 2^8
 constexpr float kNegSentinel = -1.0e30f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Schedule shared by the main and the combine kernel (lives in the workspace).
+// Pairs are ordered longest probe first: pair = (P-1-j) * B + b.  Every pair owns
+// nl * Hkv units (layer, kv head) of n_su tiles each: n_ctx context tiles followed by
+// n_own tiles of the probe's own tokens.
+struct Sched {
+  long long total;                   // tiles of all units
+  long long per;                     // tiles per gang range
+  long long prefix[kMaxPairs + 1];   // first tile of every pair in the global sequence
+  long long Lj[kMaxPairs];           // context length of the pair's probe (clamped to ctx_cap)
+  int n_ctx[kMaxPairs];
+  int n_su[kMaxPairs];
+};
 
 struct AttnParams {
-  const long long* ctx_off;   // [B][k+1]
-  float* o_part;              // [items][128][D] fp32, un-normalised
-  float* ml_part;             // [items][128][2]  (running max in log2 units, row sum)
+  const Sched* sched;
+  float* o_part;              // [slots][2][128][D] fp32, un-normalised
+  float* ml_part;             // [slots][2][128][2]  (running max in log2 units, row sum)
+  __nv_bfloat16* out;         // [B][nl][P][Tq][Hq][D]
+  float* lse;                 // [B][nl][P][Hq][Tq] or null
   int32_t* status;
-  long long ctx_cap;
-  int B, k, P, Tq, Hq, Hkv, G, nl;
-  int n_mt, n_chunks, tiles_per_chunk;
+  int B, P, Tq, Hq, Hkv, G, nl;
+  int n_mt, n_mp, gang, n_gangs;
   float scale_log2;           // softmax_scale * log2(e)
-  int nshots[kMaxProbes];
 };
 
 struct PrepParams {
@@ -47,7 +71,9 @@ struct PrepParams {
   __nv_bfloat16* q_rot;       // [B*nl*P*Hkv][Tq*G][D]
   __nv_bfloat16* kq_rot;      // layout of kq
   const long long* ctx_off;
-  int B, k, P, Tq, Hq, Hkv, nl;
+  Sched* sched;
+  long long ctx_cap;
+  int B, k, P, Tq, Hq, Hkv, nl, n_gangs;
   double rope_base;
   int nshots[kMaxProbes];
 };
@@ -75,13 +101,39 @@ __device__ __forceinline__ uint4 bf16x8_pack(const float* x) {
 }
 
 // One warp per probe token (b, l, j, t): all Hq query heads and Hkv key heads of the
-// token rotate by the same angles (L_j + t) * theta_i.
+// token rotate by the same angles (L_j + t) * theta_i.  Block 0 also writes the schedule.
 template <int D>
 __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   constexpr int VPH = D / 8, HALF_V = VPH / 2;
   const int lane = threadIdx.x & 31;
   __shared__ double theta_sh[D / 2];   // theta_i once per CTA: fp64 pow is slow
   if (threadIdx.x < D / 2) theta_sh[threadIdx.x] = pow(p.rope_base, -2.0 * (double)threadIdx.x / (double)D);
+
+  if (blockIdx.x == 0) {
+    Sched* sc = p.sched;
+    const int n_pairs = p.P * p.B;
+    const int n_own = (p.Tq + kTileN - 1) / kTileN;
+    for (int pi = threadIdx.x; pi < n_pairs; pi += blockDim.x) {
+      const int j = p.P - 1 - pi / p.B, b = pi % p.B;
+      long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
+      Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
+      const int n_ctx = (int)((Lj + kTileN - 1) / kTileN);
+      sc->Lj[pi] = Lj;
+      sc->n_ctx[pi] = n_ctx;
+      sc->n_su[pi] = n_ctx + n_own;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      long long acc = 0;
+      for (int pi = 0; pi < n_pairs; ++pi) {
+        sc->prefix[pi] = acc;
+        acc += (long long)sc->n_su[pi] * p.nl * p.Hkv;
+      }
+      sc->prefix[n_pairs] = acc;
+      sc->total = acc;
+      sc->per = (acc + p.n_gangs - 1) / p.n_gangs;
+    }
+  }
   __syncthreads();
   const long long tok = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long n_tok = (long long)p.B * p.nl * p.P * p.Tq;
@@ -130,78 +182,102 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   }
 }
 
-constexpr int kMaxPairs = 256;       // (probe, query) pairs one call may hold: B * P <= 256
-
 // Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
 template <int D>
 struct AttnSmem {
-  static constexpr int kKStages = D == 128 ? 2 : 3;
+  static constexpr int kKStages = 2;
   static constexpr int kVStages = 3;
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
-  static constexpr uint32_t kOffQ = 0;                                    // 2 buffers
+  static constexpr uint32_t kOffQ = 0;                                    // Q of M tile A, then of M tile B
   static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
   static constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
   static constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
-  static constexpr uint32_t kOffPairs = kOffBar + 256;
-  static constexpr uint32_t kTotal = kOffPairs + (kMaxPairs + 1) * 4 + 1024;   // + alignment slack
+  static constexpr uint32_t kTotal = kOffBar + 512 + 1024;               // barriers + alignment slack
 };
 
 // mbarrier slots (8 bytes each)
 enum Bar {
   kBarQFull = 0, kBarQEmpty = 2, kBarKFull = 4, kBarKEmpty = 7, kBarVFull = 10, kBarVEmpty = 13,
-  kBarSFull = 16, kBarPFull = 18, kBarPVDone = 20, kBarOFull = 21, kBarOEmpty = 23, kBarDrain = 25,
-  kNumBars = 26
+  kBarSFull = 16, kBarPFull = 18, kBarOFull = 20, kBarOEmpty = 22, kBarDrain = 24,
+  kNumBars = 25
 };
 
-struct WorkItem {
-  int b, l, j, g, mt, c;
+// A piece = the part of one unit (pair, layer, kv head) that falls into a gang's range.
+struct Piece {
+  int pair, su, t0, t1, n_su, n_ctx;
   long long Lj;
-  int t_begin, n_ctx, n_own, n_tiles;
-  int outer_ctx, outer_own, outer_q;
-  long long item_out;
+  bool first_of_gang;
 };
 
-// idx-th non-empty piece of work.  prefix[pi] = first index of pair pi = jj * B + b,
-// jj = P-1-j (longest probes first); inside a pair: chunk, layer, kv head, M tile
-// (M tile fastest, so CTAs that share a K/V chunk run at the same time).
-__device__ __forceinline__ void decode_item(const AttnParams& p, const int* prefix, int n_pairs, int idx,
-                                            WorkItem& w) {
+struct Walker {
+  long long x, begin, end;
+};
+
+__device__ __forceinline__ int find_pair(const Sched* sc, int n_pairs, long long x) {
   int lo = 0, hi = n_pairs;
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (prefix[mid] <= idx) lo = mid; else hi = mid;
+    if (sc->prefix[mid] <= x) lo = mid; else hi = mid;
   }
-  int local = idx - prefix[lo];
-  w.j = p.P - 1 - lo / p.B;
-  w.b = lo % p.B;
-  w.mt = local % p.n_mt; local /= p.n_mt;
-  w.g = local % p.Hkv; local /= p.Hkv;
-  w.l = local % p.nl;
-  w.c = local / p.nl;
-  long long Lj = p.ctx_off[(long long)w.b * (p.k + 1) + p.nshots[w.j]];
-  Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
-  w.Lj = Lj;
-  const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
-  const int c_last = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk : 0;
-  w.t_begin = w.c * p.tiles_per_chunk;
-  w.n_ctx = max(0, min(n_tiles_ctx, w.t_begin + p.tiles_per_chunk) - w.t_begin);
-  w.n_own = 0;
-  if (w.c == c_last) {   // the last chunk also takes the probe's own tokens (causal part)
-    const int row_hi = min(p.Tq * p.G - 1, w.mt * kTileM + kTileM - 1);
-    w.n_own = (row_hi / p.G) / kTileN + 1;
-  }
+  return lo;
+}
+
+__device__ __forceinline__ bool next_piece(const Sched* sc, int n_pairs, Walker& wk, Piece& pc) {
+  if (wk.x >= wk.end) return false;
+  const int lo = find_pair(sc, n_pairs, wk.x);
+  const int nsu = sc->n_su[lo];
+  const long long rel = wk.x - sc->prefix[lo];
+  pc.pair = lo;
+  pc.su = (int)(rel / nsu);
+  pc.t0 = (int)(rel % nsu);
+  const long long room = wk.end - wk.x;
+  pc.t1 = (int)(room < (long long)(nsu - pc.t0) ? pc.t0 + room : nsu);
+  pc.n_su = nsu;
+  pc.n_ctx = sc->n_ctx[lo];
+  pc.Lj = sc->Lj[lo];
+  pc.first_of_gang = wk.x == wk.begin;
+  wk.x += pc.t1 - pc.t0;
+  return true;
+}
+
+// One M pair of one piece: what a CTA works on between two read-outs of O.
+struct Item {
+  int b, l, j, g, mp;
+  bool has_b, whole;
+  int ctx_begin, n_ctx, own_begin, n_own, n_tiles;
+  long long Lj;
+  int outer_ctx, outer_own, outer_q;
+  long long slot;
+};
+
+__device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, int gang_id, int mp, Item& w) {
+  w.j = p.P - 1 - pc.pair / p.B;
+  w.b = pc.pair % p.B;
+  w.l = pc.su / p.Hkv;
+  w.g = pc.su % p.Hkv;
+  w.mp = mp;
+  w.has_b = 2 * mp + 1 < p.n_mt;
+  w.whole = pc.t0 == 0 && pc.t1 == pc.n_su;
+  w.Lj = pc.Lj;
+  const int ctx_end = min(pc.t1, pc.n_ctx);
+  w.ctx_begin = pc.t0;
+  w.n_ctx = max(0, ctx_end - pc.t0);
+  // own-token tiles this M pair can see (causal): tokens up to the pair's last row
+  const int row_hi = min(p.Tq * p.G - 1, mp * 2 * kTileM + 2 * kTileM - 1);
+  const int own_need = (row_hi / p.G) / kTileN + 1;
+  w.own_begin = max(pc.t0, pc.n_ctx) - pc.n_ctx;
+  const int own_end = min(pc.t1 - pc.n_ctx, own_need);
+  w.n_own = max(0, own_end - w.own_begin);
   w.n_tiles = w.n_ctx + w.n_own;
   w.outer_ctx = w.b * p.nl + w.l;
   w.outer_own = w.outer_ctx * p.P + w.j;
   w.outer_q = w.outer_own * p.Hkv + w.g;
-  w.item_out = (((long long)w.outer_own * p.Hkv + w.g) * p.n_mt + w.mt) * p.n_chunks + w.c;
+  w.slot = ((long long)(2 * gang_id + (pc.first_of_gang ? 0 : 1)) * p.n_mp + mp);
 }
 
-// Persistent kernel: one CTA per SM walks over the non-empty work items round-robin.
-// TMEM: S/P buffers at columns 0 and 128 (P, as packed bf16, overwrites the S tile it
-// was computed from), O accumulators at 256 and 384 (alternating per item so that the
-// read-out of one item overlaps the MMAs of the next).
+// TMEM: S/P of M tile A at columns 0..127, of M tile B at 128..255 (P, as packed bf16,
+// overwrites the S tile it was computed from); O accumulators at 256 and 384.
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
@@ -223,21 +299,12 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   auto bar = [&](int i) { return bar0 + 8u * i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + SM::kOffBar + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + SM::kOffBar + 8 * kNumBars + 8);
-  int* prefix = reinterpret_cast<int*>(base_ptr + SM::kOffPairs);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_pairs = p.P * p.B;
+  const int gang_id = blockIdx.x / p.gang, rank = blockIdx.x % p.gang;
+  const Sched* sc = p.sched;
 
-  // ---- how many non-empty items every (probe, query) pair has
-  const int per_chunk = p.nl * p.Hkv * p.n_mt;
-  for (int pi = threadIdx.x; pi < n_pairs; pi += kAttnThreads) {
-    const int j = p.P - 1 - pi / p.B, b = pi % p.B;
-    long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
-    Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
-    const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
-    const int n_valid = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk + 1 : 1;
-    prefix[pi + 1] = n_valid * per_chunk;
-  }
   if (threadIdx.x == 32) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(kBarQFull + i), 1);
@@ -253,7 +320,6 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       mbar_init(bar(kBarVFull + i), 1);
       mbar_init(bar(kBarVEmpty + i), 1);
     }
-    mbar_init(bar(kBarPVDone), 1);
     mbar_init(bar(kBarDrain), 1);
     abort_flag[0] = 0;
     abort_flag[1] = 0;
@@ -265,57 +331,62 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) {
-    prefix[0] = 0;
-    for (int pi = 0; pi < n_pairs; ++pi) prefix[pi + 1] += prefix[pi];
-  }
-  __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total = prefix[n_pairs];
+
+  Walker wk0;
+  wk0.begin = (long long)gang_id * sc->per;
+  wk0.end = wk0.begin + sc->per < sc->total ? wk0.begin + sc->per : sc->total;
+  wk0.x = wk0.begin;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_kctx); tma_prefetch_desc(&tm_vctx);
-      uint32_t tk = 0, tv = 0;
-      int n = 0;
+      uint32_t tk = 0, tv = 0, nq[2] = {0, 0};
       bool ok = true;
-      for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
-        WorkItem w;
-        decode_item(p, prefix, n_pairs, idx, w);
-        const int qb = n & 1;
-        ok = mbar_wait(bar(kBarQEmpty + qb), ((n >> 1) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar(kBarQFull + qb), kTileBytes);
+      Walker wk = wk0;
+      Piece pc;
+      while (ok && next_piece(sc, n_pairs, wk, pc)) {
+        for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
+          Item w;
+          make_item(p, pc, gang_id, mp, w);
+          if (w.n_tiles == 0) continue;
+          for (int x = 0; x < (w.has_b ? 2 : 1) && ok; ++x) {
+            ok = mbar_wait(bar(kBarQEmpty + x), (nq[x] & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar(kBarQFull + x), kTileBytes);
 #pragma unroll
-        for (int s = 0; s < SUB; ++s)
-          tma_load_3d(base + SM::kOffQ + qb * kTileBytes + s * 16384u, &tm_q, bar(kBarQFull + qb), s * 64,
-                      w.mt * kTileM, w.outer_q);
-        for (int i = 0; i < w.n_tiles; ++i) {
-          const bool own = i >= w.n_ctx;
-          const CUtensorMap* mk = own ? &tm_kown : &tm_kctx;
-          const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
-          const int row = own ? (i - w.n_ctx) * kTileN : (w.t_begin + i) * kTileN;
-          const int outer = own ? w.outer_own : w.outer_ctx;
-          const int sk = tk % KS;
-          ok = mbar_wait(bar(kBarKEmpty + sk), ((tk / KS) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar(kBarKFull + sk), kTileBytes);
+            for (int s = 0; s < SUB; ++s)
+              tma_load_3d(base + SM::kOffQ + x * kTileBytes + s * 16384u, &tm_q, bar(kBarQFull + x), s * 64,
+                          (2 * mp + x) * kTileM, w.outer_q);
+            ++nq[x];
+          }
+          for (int i = 0; i < w.n_tiles && ok; ++i) {
+            const bool own = i >= w.n_ctx;
+            const CUtensorMap* mk = own ? &tm_kown : &tm_kctx;
+            const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
+            const int row = own ? (w.own_begin + i - w.n_ctx) * kTileN : (w.ctx_begin + i) * kTileN;
+            const int outer = own ? w.outer_own : w.outer_ctx;
+            const int sk = tk % KS;
+            ok = mbar_wait(bar(kBarKEmpty + sk), ((tk / KS) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar(kBarKFull + sk), kTileBytes);
 #pragma unroll
-          for (int s = 0; s < SUB; ++s)
-            tma_load_4d(base + SM::kOffK + sk * kTileBytes + s * 16384u, mk, bar(kBarKFull + sk), s * 64, w.g, row,
-                        outer);
-          ++tk;
-          const int sv = tv % VS;
-          ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
+            for (int s = 0; s < SUB; ++s)
+              tma_load_4d(base + SM::kOffK + sk * kTileBytes + s * 16384u, mk, bar(kBarKFull + sk), s * 64, w.g, row,
+                          outer);
+            ++tk;
+            const int sv = tv % VS;
+            ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
 #pragma unroll
-          for (int s = 0; s < SUB; ++s)
-            tma_load_4d(base + SM::kOffV + sv * kTileBytes + s * 16384u, mv, bar(kBarVFull + sv), s * 64, w.g, row,
-                        outer);
-          ++tv;
+            for (int s = 0; s < SUB; ++s)
+              tma_load_4d(base + SM::kOffV + sv * kTileBytes + s * 16384u, mv, bar(kBarVFull + sv), s * 64, w.g, row,
+                          outer);
+            ++tv;
+          }
         }
       }
       if (!ok) {
@@ -324,66 +395,87 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           mbar_wait(bar(kBarKFull + t % KS), (t / KS) & 1, abort_flag + 1);
         for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
           mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
-        for (int t = max(0, n - 1); t <= n; ++t)
-          mbar_wait(bar(kBarQFull + (t & 1)), (t >> 1) & 1, abort_flag + 1);
+        for (int x = 0; x < 2; ++x)
+          if (nq[x] > 0) mbar_wait(bar(kBarQFull + x), (nq[x] - 1) & 1, abort_flag + 1);
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      struct Pending { int sb, sv, vphase, pphase, ob, ophase, first, last; };
-      Pending prev{};
-      bool have_prev = false, ok = true;
-      auto issue_pv = [&](const Pending& t) -> bool {
-        if (t.first && !mbar_wait(bar(kBarOEmpty + t.ob), t.ophase ^ 1, abort_flag)) return false;
-        if (!mbar_wait(bar(kBarPFull + t.sb), t.pphase, abort_flag)) return false;
-        if (!mbar_wait(bar(kBarVFull + t.sv), t.vphase, abort_flag)) return false;
-        tc_fence_after();
-        const uint32_t v_base = base + SM::kOffV + t.sv * kTileBytes;
+      uint32_t tk = 0, tv = 0, np[2] = {0, 0}, ni[2] = {0, 0};
+      bool ok = true;
+      Walker wk = wk0;
+      Piece pc;
+      auto issue_qk = [&](int x, uint32_t k_base) {
+        const uint32_t q_base = base + SM::kOffQ + x * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t o = (ks / 4) * 16384u + (ks % 4) * 32u;
+          umma_ss(tmem_base + kTmemS + x * kTileN, smem_desc_sw128(q_base + o, 16, 1024),
+                  smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar(kBarSFull + x));
+      };
+      auto issue_pv = [&](int x, uint32_t v_base, bool first) {
 #pragma unroll
         for (int ks = 0; ks < kTileN / 16; ++ks) {
           // A = P from TMEM: 16 bf16 keys of one k-step occupy 8 packed columns
-          umma_ts(tmem_base + kTmemO + t.ob * 128, tmem_base + kTmemS + t.sb * kTileN + ks * 8,
-                  smem_desc_sw128(v_base + ks * 2048u, 16384, 1024), kIdescPV, (!t.first || ks > 0) ? 1u : 0u);
+          umma_ts(tmem_base + kTmemO + x * 128, tmem_base + kTmemS + x * kTileN + ks * 8,
+                  smem_desc_sw128(v_base + ks * 2048u, 16384, 1024), kIdescPV, (!first || ks > 0) ? 1u : 0u);
         }
-        umma_commit(bar(kBarVEmpty + t.sv));
-        umma_commit(bar(kBarPVDone));
-        if (t.last) umma_commit(bar(kBarOFull + t.ob));
-        return true;
       };
-      uint32_t tk = 0, tv = 0, gt = 0;
-      int n = 0;
-      for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
-        WorkItem w;
-        decode_item(p, prefix, n_pairs, idx, w);
-        const int qb = n & 1;
-        ok = mbar_wait(bar(kBarQFull + qb), (n >> 1) & 1, abort_flag);
-        const uint32_t q_base = base + SM::kOffQ + qb * kTileBytes;
-        for (int i = 0; i < w.n_tiles && ok; ++i) {
-          const int sk = tk % KS, sb = gt & 1;
-          ok = mbar_wait(bar(kBarKFull + sk), (tk / KS) & 1, abort_flag);
+      while (ok && next_piece(sc, n_pairs, wk, pc)) {
+        for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
+          Item w;
+          make_item(p, pc, gang_id, mp, w);
+          if (w.n_tiles == 0) continue;
+          const int nx = w.has_b ? 2 : 1;
+          // S of the first tile for both M tiles
+          for (int x = 0; x < nx && ok; ++x) ok = mbar_wait(bar(kBarQFull + x), ni[x] & 1, abort_flag);
+          if (!ok) break;
+          ok = mbar_wait(bar(kBarKFull + tk % KS), (tk / KS) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t k_base = base + SM::kOffK + sk * kTileBytes;
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t o = (ks / 4) * 16384u + (ks % 4) * 32u;
-            umma_ss(tmem_base + kTmemS + sb * kTileN, smem_desc_sw128(q_base + o, 16, 1024),
-                    smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+          for (int x = 0; x < nx; ++x) {
+            issue_qk(x, base + SM::kOffK + (tk % KS) * kTileBytes);
+            if (w.n_tiles == 1) umma_commit(bar(kBarQEmpty + x));
           }
-          umma_commit(bar(kBarSFull + sb));
-          umma_commit(bar(kBarKEmpty + sk));
-          if (i == w.n_tiles - 1) umma_commit(bar(kBarQEmpty + qb));
+          umma_commit(bar(kBarKEmpty + tk % KS));
           ++tk;
-          if (have_prev) ok = issue_pv(prev);
-          prev.sb = sb; prev.sv = tv % VS; prev.vphase = (tv / VS) & 1; prev.pphase = (gt >> 1) & 1;
-          prev.ob = n & 1; prev.ophase = (n >> 1) & 1; prev.first = i == 0; prev.last = i == w.n_tiles - 1;
-          have_prev = true;
-          ++tv; ++gt;
+          for (int i = 0; i < w.n_tiles && ok; ++i) {
+            const bool next = i + 1 < w.n_tiles;
+            const uint32_t k_base = base + SM::kOffK + (tk % KS) * kTileBytes;
+            const uint32_t v_base = base + SM::kOffV + (tv % VS) * kTileBytes;
+            if (next) ok = mbar_wait(bar(kBarKFull + tk % KS), (tk / KS) & 1, abort_flag);
+            if (ok) ok = mbar_wait(bar(kBarVFull + tv % VS), (tv / VS) & 1, abort_flag);
+            for (int x = 0; x < nx && ok; ++x) {
+              // O of the previous item must have been read out before the first PV overwrites it
+              if (i == 0) ok = mbar_wait(bar(kBarOEmpty + x), (ni[x] & 1) ^ 1, abort_flag);
+              if (ok) ok = mbar_wait(bar(kBarPFull + x), np[x] & 1, abort_flag);
+              if (!ok) break;
+              ++np[x];
+              tc_fence_after();
+              issue_pv(x, v_base, i == 0);
+              if (next) {
+                // S(i+1) overwrites P(i) in place: the tensor pipe runs its operations in order
+                issue_qk(x, k_base);
+                if (i + 2 == w.n_tiles) umma_commit(bar(kBarQEmpty + x));
+              } else {
+                umma_commit(bar(kBarOFull + x));
+              }
+            }
+            if (!ok) break;
+            umma_commit(bar(kBarVEmpty + tv % VS));
+            ++tv;
+            if (next) {
+              umma_commit(bar(kBarKEmpty + tk % KS));
+              ++tk;
+            }
+          }
+          for (int x = 0; x < nx; ++x) ++ni[x];
         }
       }
-      if (ok && have_prev) ok = issue_pv(prev);
       if (!ok) {
         umma_commit(bar(kBarDrain));
         mbar_wait(bar(kBarDrain), 0, abort_flag + 1);
@@ -391,108 +483,152 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     __syncwarp();
   } else {
-    // ---------------------------------------------------- softmax + correction
+    // ---------------------------------------------------- softmax + read-out of O
+    const int x = (warp - 2) >> 2;                 // 0: M tile A, 1: M tile B
     const int quarter = warp & 3;                  // TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;             // row of the M tile
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    uint32_t gt = 0;
-    int n = 0;
+    const uint32_t s_addr = tmem_base + lane_addr + kTmemS + x * kTileN;
+    const uint32_t o_addr = tmem_base + lane_addr + kTmemO + x * 128;
+    uint32_t ns = 0, ni = 0;
     bool ok = true;
-    for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++n) {
-      WorkItem w;
-      decode_item(p, prefix, n_pairs, idx, w);
-      const int ob = n & 1;
-      const int t_row = (w.mt * kTileM + r) / p.G;   // probe token of this row
-      float m_used = kNegSentinel, l_sum = 0.f;
-      for (int i = 0; i < w.n_tiles; ++i, ++gt) {
-        const int sb = gt & 1;
-        const uint32_t s_addr = tmem_base + lane_addr + kTmemS + sb * kTileN;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + sb), (gt >> 1) & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        float s[kTileN];
-        tmem_ld128(s_addr, reinterpret_cast<uint32_t*>(s));
-
-        // mask: context keys at or beyond L_j; own keys after the row's token (causal).
-        // Only the last context tile and the own-token tiles can hide anything.
-        int limit = kTileN;                          // columns < limit are visible
-        if (i < w.n_ctx) {
-          const long long first = (long long)(w.t_begin + i) * kTileN;
-          if (first + kTileN > w.Lj) limit = (int)(w.Lj - first);
-        } else {
-          limit = min(t_row, p.Tq - 1) - (i - w.n_ctx) * kTileN + 1;   // <= 0: the whole tile is hidden
-        }
-        if (__any_sync(0xffffffffu, limit < kTileN)) {
-#pragma unroll
-          for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
-        }
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int cidx = 0; cidx < kTileN; cidx += 8) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) mx[u] = fmax3(mx[u], s[cidx + 2 * u], s[cidx + 2 * u + 1]);
-        }
-        const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
-        float alpha = 1.f;
-        const bool need = tile_max > m_used + kRescaleThreshold;
-        if (need) {
-          alpha = exp2f(m_used - tile_max);
-          m_used = tile_max;
-          l_sum *= alpha;
-        }
-        // P = 2^(s * scale - m) as packed bf16 back into the S columns (two keys per column);
-        // scale-and-shift and the row sum run two columns per instruction (packed fp32)
-        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
-        const float2 neg_m2 = make_float2(-m_used, -m_used);
-        float2 part[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-        uint32_t pk[kTileN / 2];
-#pragma unroll
-        for (int c2 = 0; c2 < kTileN / 2; ++c2) {
-          const float2 x = __ffma2_rn(make_float2(s[2 * c2], s[2 * c2 + 1]), scale2, neg_m2);
-          const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-          part[c2 & 3] = __fadd2_rn(part[c2 & 3], e);
-          pk[c2] = pack_bf16x2(e.x, e.y);
-        }
-        const float2 tot = __fadd2_rn(__fadd2_rn(part[0], part[1]), __fadd2_rn(part[2], part[3]));
-        l_sum += tot.x + tot.y;
-        tmem_st64(s_addr, pk);
-        if (i > 0 && __any_sync(0xffffffffu, need)) {
-          // O may only be rescaled between PV(i-1) and PV(i).  PV(i) cannot start before this
-          // thread has arrived on PFull below, so the barrier is never more than one phase ahead.
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarPVDone), (gt - 1) & 1, abort_flag));
+    Walker wk = wk0;
+    Piece pc;
+    while (ok && next_piece(sc, n_pairs, wk, pc)) {
+      for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
+        Item w;
+        make_item(p, pc, gang_id, mp, w);
+        if (x == 1 && !w.has_b) continue;
+        const int mt = 2 * mp + x;
+        const int m = mt * kTileM + r;               // row of the unit: token m / G, head m % G
+        const int t_row = m / p.G;
+        float m_used = kNegSentinel, l_sum = 0.f;
+        for (int i = 0; i < w.n_tiles; ++i, ++ns) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + x), ns & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
+          float s[kTileN];
+          tmem_ld128(s_addr, reinterpret_cast<uint32_t*>(s));
+
+          // mask: context keys at or beyond L_j; own keys after the row's token (causal).
+          // Only the last context tile and the own-token tiles can hide anything.
+          int limit = kTileN;                          // columns < limit are visible
+          if (i < w.n_ctx) {
+            const long long first = (long long)(w.ctx_begin + i) * kTileN;
+            if (first + kTileN > w.Lj) limit = (int)(w.Lj - first);
+          } else {
+            limit = min(t_row, p.Tq - 1) - (w.own_begin + i - w.n_ctx) * kTileN + 1;   // <= 0: all hidden
+          }
+          if (__any_sync(0xffffffffu, limit < kTileN)) {
+#pragma unroll
+            for (int cidx = 0; cidx < kTileN; ++cidx) s[cidx] = cidx < limit ? s[cidx] : -INFINITY;
+          }
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int cidx = 0; cidx < kTileN; cidx += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) mx[u] = fmax3(mx[u], s[cidx + 2 * u], s[cidx + 2 * u + 1]);
+          }
+          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;
+          float alpha = 1.f;
+          const bool need = tile_max > m_used + kRescaleThreshold;
+          if (need) {
+            alpha = exp2f(m_used - tile_max);
+            m_used = tile_max;
+            l_sum *= alpha;
+          }
+          // P = 2^(s * scale - m) as packed bf16 back into the S columns (two keys per column);
+          // scale-and-shift and the row sum run two columns per instruction (packed fp32)
+          const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+          const float2 neg_m2 = make_float2(-m_used, -m_used);
+          float2 part[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+          uint32_t pk[kTileN / 2];
+#pragma unroll
+          for (int c2 = 0; c2 < kTileN / 2; ++c2) {
+            const float2 xs = __ffma2_rn(make_float2(s[2 * c2], s[2 * c2 + 1]), scale2, neg_m2);
+            const float2 e = make_float2(ex2_approx(xs.x), ex2_approx(xs.y));
+            part[c2 & 3] = __fadd2_rn(part[c2 & 3], e);
+            pk[c2] = pack_bf16x2(e.x, e.y);
+          }
+          const float2 tot = __fadd2_rn(__fadd2_rn(part[0], part[1]), __fadd2_rn(part[2], part[3]));
+          l_sum += tot.x + tot.y;
+          tmem_st64(s_addr, pk);
+          if (i > 0 && __any_sync(0xffffffffu, need)) {
+            // S(i) is complete, so PV(i-1), issued before it, is complete too; PV(i) waits for
+            // the arrival below: O is quiescent here.
+#pragma unroll
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+              float o[32];
+              tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] *= alpha;
+              tmem_st32(o_addr + q4 * 32, reinterpret_cast<const uint32_t*>(o));
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(bar(kBarPFull + x));
+        }
+        if (!ok) break;
+        const bool row_ok = m < p.Tq * p.G;
+        if (w.n_tiles == 0) {
+          // nothing of this M pair falls into the piece: a neutral partial (a whole unit is never empty)
+          if (row_ok) {
+            float* orow = p.o_part + ((w.slot * 2 + x) * kTileM + r) * D;
+#pragma unroll
+            for (int e = 0; e < D; e += 4) *reinterpret_cast<float4*>(orow + e) = make_float4(0.f, 0.f, 0.f, 0.f);
+            float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
+            ml[0] = kNegSentinel;
+            ml[1] = 0.f;
+          }
+          continue;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + x), ni & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (w.whole) {
+          // the piece covers the unit: normalise and store the final rows
+          const float inv = 1.f / l_sum;
+          const int t = t_row, hh = m % p.G, h = w.g * p.G + hh;
+          const long long bpj = w.outer_own;
+          __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D;
 #pragma unroll
           for (int q4 = 0; q4 < D / 32; ++q4) {
             float o[32];
-            const uint32_t addr = tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32;
-            tmem_ld32(addr, reinterpret_cast<uint32_t*>(o));
+            tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
+            if (row_ok) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] *= alpha;
-            tmem_st32(addr, reinterpret_cast<const uint32_t*>(o));
+              for (int e = 0; e < 32; e += 8) {
+                float v8[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v8[u] = o[e + u] * inv;
+                *reinterpret_cast<uint4*>(dst + q4 * 32 + e) = bf16x8_pack(v8);
+              }
+            }
+          }
+          if (row_ok && p.lse != nullptr)
+            p.lse[(bpj * p.Hq + h) * p.Tq + t] = (m_used + log2f(l_sum)) * kLn2;
+        } else {
+          float* orow = p.o_part + ((w.slot * 2 + x) * kTileM + r) * D;
+#pragma unroll
+          for (int q4 = 0; q4 < D / 32; ++q4) {
+            float o[32];
+            tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
+            if (row_ok) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<float4*>(orow + q4 * 32 + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+            }
+          }
+          if (row_ok) {
+            float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
+            ml[0] = m_used;
+            ml[1] = l_sum;
           }
         }
         tc_fence_before();
-        mbar_arrive(bar(kBarPFull + sb));
+        mbar_arrive(bar(kBarOEmpty + x));
+        ++ni;
       }
-      if (!ok) break;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + ob), (n >> 1) & 1, abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      float* orow = p.o_part + (w.item_out * kTileM + r) * D;
-#pragma unroll
-      for (int q4 = 0; q4 < D / 32; ++q4) {
-        float o[32];
-        tmem_ld32(tmem_base + lane_addr + kTmemO + ob * 128 + q4 * 32, reinterpret_cast<uint32_t*>(o));
-#pragma unroll
-        for (int e = 0; e < 32; e += 4)
-          *reinterpret_cast<float4*>(orow + q4 * 32 + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-      }
-      tc_fence_before();
-      mbar_arrive(bar(kBarOEmpty + ob));
-      float* ml = p.ml_part + (w.item_out * kTileM + r) * 2;
-      ml[0] = m_used;
-      ml[1] = l_sum;
     }
   }
 
@@ -506,59 +642,68 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 }
 
 struct CombineParams {
-  const long long* ctx_off;
+  const Sched* sched;
   const float* o_part;
   const float* ml_part;
   __nv_bfloat16* out;   // [B][nl][P][Tq][Hq][D]
   float* lse;           // [B][nl][P][Hq][Tq] or null
-  long long ctx_cap;
-  int B, k, P, Tq, Hq, Hkv, G, nl, n_mt, n_chunks, tiles_per_chunk;
-  int nshots[kMaxProbes];
+  int B, P, Tq, Hq, Hkv, G, nl, n_mp, n_gangs;
 };
 
-// One warp per output row (b, l, j, t, h): merge the chunk partials.
+// Block (q, y): if the range of gang q ends inside a unit that starts in that range, the
+// unit was cut; its pieces sit with gangs q .. q_last.  One warp merges one row.
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p) {
+  const Sched* sc = p.sched;
+  const int q = blockIdx.x;
+  const long long per = sc->per, total = sc->total;
+  const long long cut = (long long)(q + 1) * per;
+  if (per <= 0 || cut >= total) return;
+  const int n_pairs = p.P * p.B;
+  const int pair = find_pair(sc, n_pairs, cut);
+  const int nsu = sc->n_su[pair];
+  const long long rel = cut - sc->prefix[pair];
+  if (rel % nsu == 0) return;                       // the cut falls between two units
+  const int su = (int)(rel / nsu);
+  const long long s_u = sc->prefix[pair] + (long long)su * nsu, e_u = s_u + nsu;
+  if (s_u < (long long)q * per) return;             // an earlier gang holds the unit's first piece
+  const int q_last = (int)((e_u - 1) / per);
+
   const int lane = threadIdx.x & 31;
-  const long long row_id = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long n_rows = (long long)p.B * p.nl * p.P * p.Tq * p.Hq;
-  if (row_id >= n_rows) return;
-  const int h = (int)(row_id % p.Hq);
-  const int t = (int)((row_id / p.Hq) % p.Tq);
-  const long long bpj = row_id / ((long long)p.Hq * p.Tq);
-  const int j = (int)(bpj % p.P);
-  const int b = (int)(bpj / ((long long)p.P * p.nl));
-  const int g = h / p.G, hh = h % p.G;
-  const int m = t * p.G + hh, mt = m / kTileM, r = m % kTileM;
+  const int m = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (m >= p.Tq * p.G) return;
+  const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
+  const int j = p.P - 1 - pair / p.B, b = pair % p.B;
+  const int l = su / p.Hkv, g = su % p.Hkv;
+  const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
+  const long long bpj = ((long long)b * p.nl + l) * p.P + j;
 
-  long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
-  Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
-  const int n_tiles_ctx = (int)((Lj + kTileN - 1) / kTileN);
-  const int c_last = n_tiles_ctx > 0 ? (n_tiles_ctx - 1) / p.tiles_per_chunk : 0;
-  const long long item0 = ((bpj * p.Hkv + g) * p.n_mt + mt) * (long long)p.n_chunks;
-
+  auto slot_row = [&](int qq) -> long long {
+    const int which = (long long)qq * per >= s_u ? 0 : 1;   // the gang's first piece, or its last
+    return (((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x) * kTileM + r;
+  };
   float M = kNegSentinel;
-  for (int c = 0; c <= c_last; ++c) M = fmaxf(M, p.ml_part[((item0 + c) * kTileM + r) * 2]);
+  for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[slot_row(qq) * 2]);
   constexpr int EPL = D / 32;                      // output elements per lane
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   float lsum = 0.f;
-  for (int c = 0; c <= c_last; ++c) {
-    const float* ml = p.ml_part + ((item0 + c) * kTileM + r) * 2;
-    const float w = exp2f(ml[0] - M);
-    lsum += ml[1] * w;
-    const float* o = p.o_part + ((item0 + c) * kTileM + r) * D + lane * EPL;
+  for (int qq = q; qq <= q_last; ++qq) {
+    const long long sr = slot_row(qq);
+    const float wgt = exp2f(p.ml_part[sr * 2] - M);
+    lsum += p.ml_part[sr * 2 + 1] * wgt;
+    const float* o = p.o_part + sr * D + lane * EPL;
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] += o[e] * w;
+    for (int e = 0; e < EPL; ++e) acc[e] += o[e] * wgt;
   }
   const float inv = 1.f / lsum;
-  __nv_bfloat16* dst = p.out + row_id * D + lane * EPL;
+  __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D + lane * EPL;
 #pragma unroll
   for (int e = 0; e < EPL; e += 2)
     *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
   if (p.lse != nullptr && lane == 0)
-    p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * 0.6931471805599453f;
+    p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * kLn2;
 }
 
 // ----------------------------------------------------------------- host side
@@ -596,36 +741,27 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 }
 
 struct AttnPlan {
-  int n_mt, n_chunks, tiles_per_chunk;
-  long long items;
-  size_t off_qrot, off_kqrot, off_opart, off_ml, total;
+  int n_mt, n_mp, gang;
+  size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, total;
 };
 
-AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, long long ctx_cap,
-                   uint32_t flags) {
+// The gang (CTAs that walk the same K/V tiles, one M pair each per round) is the number of
+// M pairs when that is at most kMaxGang, else the M pairs are dealt out in rounds.
+AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl) {
   AttnPlan pl;
   const int G = model->n_q_heads / model->n_kv_heads;
   const int D = model->head_dim;
   pl.n_mt = (Tq * G + kTileM - 1) / kTileM;
-  const long long tiles_cap = (ctx_cap + kTileN - 1) / kTileN;
-  const long long base_items = (long long)B * nl * P * model->n_kv_heads * pl.n_mt;
-  long long tpc = flags & 0xffffu;
-  if (tpc == 0) {
-    // about four waves of 148 CTAs when the context allows it, at least 8 tiles each
-    long long want = (4 * 148 + base_items - 1) / base_items;
-    tpc = (tiles_cap + want - 1) / want;
-    if (tpc < 8) tpc = 8;
-  }
-  if (tpc > tiles_cap) tpc = tiles_cap > 0 ? tiles_cap : 1;
-  pl.tiles_per_chunk = (int)tpc;
-  pl.n_chunks = (int)((tiles_cap + tpc - 1) / tpc);
-  if (pl.n_chunks < 1) pl.n_chunks = 1;
-  pl.items = base_items * pl.n_chunks;
+  pl.n_mp = (pl.n_mt + 1) / 2;
+  const int rounds = (pl.n_mp + kMaxGang - 1) / kMaxGang;
+  pl.gang = (pl.n_mp + rounds - 1) / rounds;
+  const size_t slots = (size_t)2 * kMaxCtas * pl.n_mp;     // two cut pieces per gang at most
   size_t off = 0;
   pl.off_qrot = off;  off += ads_round_up((size_t)B * nl * P * Tq * model->n_q_heads * D * 2, 256);
   pl.off_kqrot = off; off += ads_round_up((size_t)B * nl * P * Tq * model->n_kv_heads * D * 2, 256);
-  pl.off_opart = off; off += ads_round_up((size_t)pl.items * kTileM * D * 4, 256);
-  pl.off_ml = off;    off += ads_round_up((size_t)pl.items * kTileM * 2 * 4, 256);
+  pl.off_sched = off; off += ads_round_up(sizeof(Sched), 256);
+  pl.off_opart = off; off += ads_round_up(slots * 2 * kTileM * D * 4, 256);
+  pl.off_ml = off;    off += ads_round_up(slots * 2 * kTileM * 2 * 4, 256);
   pl.total = off;
   return pl;
 }
@@ -644,8 +780,18 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   unsigned char* wsb = static_cast<unsigned char*>(ws);
   __nv_bfloat16* q_rot = reinterpret_cast<__nv_bfloat16*>(wsb + pl.off_qrot);
   __nv_bfloat16* kq_rot = reinterpret_cast<__nv_bfloat16*>(wsb + pl.off_kqrot);
+  Sched* sched = reinterpret_cast<Sched*>(wsb + pl.off_sched);
   float* o_part = reinterpret_cast<float*>(wsb + pl.off_opart);
   float* ml_part = reinterpret_cast<float*>(wsb + pl.off_ml);
+
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    ADS_CHECK_CUDA(cudaGetDevice(&dev));
+    ADS_CHECK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const int n_cta = n_sm < kMaxCtas ? n_sm : kMaxCtas;
+  const int n_gangs = n_cta / pl.gang > 0 ? n_cta / pl.gang : 1;
 
   // ---- tensor maps
   CUtensorMap tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown;
@@ -670,11 +816,12 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     if (!make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
   }
 
-  // ---- rotate Q and the probe's own K
+  // ---- rotate Q and the probe's own K, write the schedule
   PrepParams pp;
   pp.q = static_cast<const __nv_bfloat16*>(q); pp.kq = static_cast<const __nv_bfloat16*>(kq);
   pp.q_rot = q_rot; pp.kq_rot = kq_rot; pp.ctx_off = reinterpret_cast<const long long*>(ctx_off);
-  pp.B = B; pp.k = k; pp.P = P; pp.Tq = Tq; pp.Hq = Hq; pp.Hkv = Hkv; pp.nl = nl;
+  pp.sched = sched; pp.ctx_cap = ctx_cap;
+  pp.B = B; pp.k = k; pp.P = P; pp.Tq = Tq; pp.Hq = Hq; pp.Hkv = Hkv; pp.nl = nl; pp.n_gangs = n_gangs;
   pp.rope_base = model->rope_base;
   for (int i = 0; i < kMaxProbes; ++i) pp.nshots[i] = i < P ? probe_nshots[i] : 0;
   const long long n_tok = (long long)B * nl * P * Tq;
@@ -683,38 +830,30 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
 
   // ---- main kernel
   AttnParams ap;
-  ap.ctx_off = reinterpret_cast<const long long*>(ctx_off);
-  ap.o_part = o_part; ap.ml_part = ml_part; ap.status = status; ap.ctx_cap = ctx_cap;
-  ap.B = B; ap.k = k; ap.P = P; ap.Tq = Tq; ap.Hq = Hq; ap.Hkv = Hkv; ap.G = G; ap.nl = nl;
-  ap.n_mt = pl.n_mt; ap.n_chunks = pl.n_chunks; ap.tiles_per_chunk = pl.tiles_per_chunk;
+  ap.sched = sched; ap.o_part = o_part; ap.ml_part = ml_part;
+  ap.out = static_cast<__nv_bfloat16*>(out); ap.lse = lse; ap.status = status;
+  ap.B = B; ap.P = P; ap.Tq = Tq; ap.Hq = Hq; ap.Hkv = Hkv; ap.G = G; ap.nl = nl;
+  ap.n_mt = pl.n_mt; ap.n_mp = pl.n_mp; ap.gang = pl.gang; ap.n_gangs = n_gangs;
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
-  for (int i = 0; i < kMaxProbes; ++i) ap.nshots[i] = pp.nshots[i];
   const int smem = (int)AttnSmem<128>::kTotal;     // same request for D = 64: one CTA per SM
   static bool attr_done[2] = {false, false};
   if (!attr_done[D == 128]) {
     ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done[D == 128] = true;
   }
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    ADS_CHECK_CUDA(cudaGetDevice(&dev));
-    ADS_CHECK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-  }
-  const unsigned grid = (unsigned)(pl.items < n_sm ? pl.items : n_sm);   // persistent: one CTA per SM
-  attn_main_kernel<D><<<grid, kAttnThreads, smem, st>>>(tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+  attn_main_kernel<D><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(tm_q, tm_kctx, tm_vctx, tm_kown,
+                                                                               tm_vown, ap);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
-  // ---- merge
+  // ---- merge the units that a range boundary cut
   CombineParams cp;
-  cp.ctx_off = ap.ctx_off; cp.o_part = o_part; cp.ml_part = ml_part;
-  cp.out = static_cast<__nv_bfloat16*>(out); cp.lse = lse; cp.ctx_cap = ctx_cap;
-  cp.B = B; cp.k = k; cp.P = P; cp.Tq = Tq; cp.Hq = Hq; cp.Hkv = Hkv; cp.G = G; cp.nl = nl;
-  cp.n_mt = pl.n_mt; cp.n_chunks = pl.n_chunks; cp.tiles_per_chunk = pl.tiles_per_chunk;
-  for (int i = 0; i < kMaxProbes; ++i) cp.nshots[i] = pp.nshots[i];
-  const long long n_rows = n_tok * Hq;
-  attn_combine_kernel<D><<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(cp);
+  cp.sched = sched; cp.o_part = o_part; cp.ml_part = ml_part;
+  cp.out = ap.out; cp.lse = lse;
+  cp.B = B; cp.P = P; cp.Tq = Tq; cp.Hq = Hq; cp.Hkv = Hkv; cp.G = G; cp.nl = nl;
+  cp.n_mp = pl.n_mp; cp.n_gangs = n_gangs;
+  const dim3 grid((unsigned)n_gangs, (unsigned)((Tq * G + 7) / 8));
+  attn_combine_kernel<D><<<grid, 256, 0, st>>>(cp);
   return ads_launch_status();
 }
 
@@ -725,10 +864,7 @@ extern "C" size_t adapshot_attn_workspace_bytes(const adapshot_model_t* model, i
   if (model == nullptr || !attn_shape_ok(model) || B <= 0 || P <= 0 || Tq <= 0 || n_layers_in_call <= 0 ||
       ctx_cap <= 0)
     return 0;
-  // sized for the finest split a caller may request through `flags`
-  AttnPlan a = make_plan(model, B, P, Tq, n_layers_in_call, ctx_cap, 0);
-  AttnPlan f = make_plan(model, B, P, Tq, n_layers_in_call, ctx_cap, 8);
-  return a.total > f.total ? a.total : f.total;
+  return make_plan(model, B, P, Tq, n_layers_in_call).total;
 }
 
 extern "C" int adapshot_query_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx,
@@ -740,7 +876,7 @@ extern "C" int adapshot_query_attn(const adapshot_model_t* model, const void* k_
   if (model == nullptr || k_ctx == nullptr || v_ctx == nullptr || ctx_off == nullptr || probe_nshots == nullptr ||
       q == nullptr || kq == nullptr || vq == nullptr || out == nullptr || ws == nullptr)
     return ADAPSHOT_EINVAL;
-  if (B <= 0 || k <= 0 || Tq <= 0 || ctx_cap <= 0 || (flags & ~0xffffu) != 0) return ADAPSHOT_EINVAL;
+  if (B <= 0 || k <= 0 || Tq <= 0 || ctx_cap <= 0 || flags != 0) return ADAPSHOT_EINVAL;
   if (model->dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
   if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
   if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
@@ -749,15 +885,13 @@ extern "C" int adapshot_query_attn(const adapshot_model_t* model, const void* k_
     if (probe_nshots[i] < 1 || probe_nshots[i] > k) return ADAPSHOT_ESHAPE;
     if (i > 0 && probe_nshots[i] <= probe_nshots[i - 1]) return ADAPSHOT_ESHAPE;
   }
-  if ((flags & 0xffffu) != 0 && (flags & 0xffffu) < 8) return ADAPSHOT_EINVAL;
   if (!ads_aligned16(k_ctx) || !ads_aligned16(v_ctx) || !ads_aligned16(q) || !ads_aligned16(kq) ||
       !ads_aligned16(vq) || !ads_aligned16(out) || ((uintptr_t)ws & 255u))
     return ADAPSHOT_EALIGN;
   if (ctx_cap > (1ll << 31) - 256) return ADAPSHOT_ESHAPE;
   const int nl = layer_end - layer_begin;
-  const AttnPlan pl = make_plan(model, B, P, Tq, nl, ctx_cap, flags);
+  const AttnPlan pl = make_plan(model, B, P, Tq, nl);
   if (ws_bytes < pl.total) return ADAPSHOT_ECAPACITY;
-  if (pl.items > 0x7fffffffll) return ADAPSHOT_ESHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (model->head_dim == 128)
     return launch_attn<128>(model, k_ctx, v_ctx, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
