@@ -403,77 +403,93 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      uint32_t tk = 0, tv = 0, np[2] = {0, 0}, ni[2] = {0, 0};
+      // The tensor pipe takes only a few UMMAs ahead of the one it runs: whatever this thread
+      // does between two issues is time the pipe may idle, so the per-tile path is kept short
+      // (scalar counters, no indexed arrays, descriptors as a constant high half plus a low
+      // half = (address >> 4) with an immediate per k-step).
+      uint32_t tk = 0, tv = 0, np0 = 0, np1 = 0, ni0 = 0, ni1 = 0;
       bool ok = true;
       Walker wk = wk0;
       Piece pc;
-      auto issue_qk = [&](int x, uint32_t k_base) {
-        const uint32_t q_base = base + SM::kOffQ + x * kTileBytes;
+      constexpr uint32_t kHi = smem_desc_hi_sw128(1024);
+      const uint32_t q_lo0 = smem_desc_lo(base + SM::kOffQ, 16);
+      const uint32_t k_lo0 = smem_desc_lo(base + SM::kOffK, 16);
+      const uint32_t v_lo0 = smem_desc_lo(base + SM::kOffV, 16384);
+      auto issue_qk = [&](const int x, uint32_t k_stage) {
+        const uint32_t q_lo = q_lo0 + x * (kTileBytes >> 4);
+        const uint32_t k_lo = k_lo0 + k_stage * (kTileBytes >> 4);
+        const uint32_t d = tmem_base + kTmemS + x * kTileN;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t o = (ks / 4) * 16384u + (ks % 4) * 32u;
-          umma_ss(tmem_base + kTmemS + x * kTileN, smem_desc_sw128(q_base + o, 16, 1024),
-                  smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+          const uint32_t o = ((ks / 4) * 16384u + (ks % 4) * 32u) >> 4;
+          umma_ss_lohi(d, q_lo + o, kHi, k_lo + o, kHi, kIdescQK, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar(kBarSFull + x));
       };
-      auto issue_pv = [&](int x, uint32_t v_base, bool first) {
+      auto issue_pv = [&](const int x, uint32_t v_stage, bool first) {
+        const uint32_t v_lo = v_lo0 + v_stage * (kTileBytes >> 4);
+        const uint32_t d = tmem_base + kTmemO + x * 128;
+        const uint32_t a = tmem_base + kTmemS + x * kTileN;
+        // A = P from TMEM: 16 bf16 keys of one k-step occupy 8 packed columns
+        umma_ts_lohi(d, a, v_lo, kHi, kIdescPV, first ? 0u : 1u);
 #pragma unroll
-        for (int ks = 0; ks < kTileN / 16; ++ks) {
-          // A = P from TMEM: 16 bf16 keys of one k-step occupy 8 packed columns
-          umma_ts(tmem_base + kTmemO + x * 128, tmem_base + kTmemS + x * kTileN + ks * 8,
-                  smem_desc_sw128(v_base + ks * 2048u, 16384, 1024), kIdescPV, (!first || ks > 0) ? 1u : 0u);
+        for (int ks = 1; ks < kTileN / 16; ++ks)
+          umma_ts_lohi(d, a + ks * 8, v_lo + ((ks * 2048u) >> 4), kHi, kIdescPV, 1u);
+      };
+      // one M tile's share of tile i: O += P V, then S of the next tile (in place of P: the
+      // tensor pipe runs its operations in order)
+      auto chain = [&](const int x, uint32_t& np_x, const uint32_t ni_x, int i, int n_tiles, uint32_t k_stage,
+                       uint32_t v_stage) -> bool {
+        // O of the previous item must have been read out before the first PV overwrites it
+        if (i == 0 && !mbar_wait(bar(kBarOEmpty + x), (ni_x & 1) ^ 1, abort_flag)) return false;
+        if (!mbar_wait(bar(kBarPFull + x), np_x & 1, abort_flag)) return false;
+        ++np_x;
+        tc_fence_after();
+        issue_pv(x, v_stage, i == 0);
+        if (i + 1 < n_tiles) {
+          issue_qk(x, k_stage);
+          if (i + 2 == n_tiles) umma_commit(bar(kBarQEmpty + x));
+        } else {
+          umma_commit(bar(kBarOFull + x));
         }
+        return true;
       };
       while (ok && next_piece(sc, n_pairs, wk, pc)) {
         for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
           Item w;
           make_item(p, pc, gang_id, mp, w);
           if (w.n_tiles == 0) continue;
-          const int nx = w.has_b ? 2 : 1;
           // S of the first tile for both M tiles
-          for (int x = 0; x < nx && ok; ++x) ok = mbar_wait(bar(kBarQFull + x), ni[x] & 1, abort_flag);
-          if (!ok) break;
-          ok = mbar_wait(bar(kBarKFull + tk % KS), (tk / KS) & 1, abort_flag);
+          ok = mbar_wait(bar(kBarQFull + 0), ni0 & 1, abort_flag);
+          if (ok && w.has_b) ok = mbar_wait(bar(kBarQFull + 1), ni1 & 1, abort_flag);
+          if (ok) ok = mbar_wait(bar(kBarKFull + tk % KS), (tk / KS) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          for (int x = 0; x < nx; ++x) {
-            issue_qk(x, base + SM::kOffK + (tk % KS) * kTileBytes);
-            if (w.n_tiles == 1) umma_commit(bar(kBarQEmpty + x));
+          issue_qk(0, tk % KS);
+          if (w.n_tiles == 1) umma_commit(bar(kBarQEmpty + 0));
+          if (w.has_b) {
+            issue_qk(1, tk % KS);
+            if (w.n_tiles == 1) umma_commit(bar(kBarQEmpty + 1));
           }
           umma_commit(bar(kBarKEmpty + tk % KS));
           ++tk;
           for (int i = 0; i < w.n_tiles && ok; ++i) {
             const bool next = i + 1 < w.n_tiles;
-            const uint32_t k_base = base + SM::kOffK + (tk % KS) * kTileBytes;
-            const uint32_t v_base = base + SM::kOffV + (tv % VS) * kTileBytes;
-            if (next) ok = mbar_wait(bar(kBarKFull + tk % KS), (tk / KS) & 1, abort_flag);
-            if (ok) ok = mbar_wait(bar(kBarVFull + tv % VS), (tv / VS) & 1, abort_flag);
-            for (int x = 0; x < nx && ok; ++x) {
-              // O of the previous item must have been read out before the first PV overwrites it
-              if (i == 0) ok = mbar_wait(bar(kBarOEmpty + x), (ni[x] & 1) ^ 1, abort_flag);
-              if (ok) ok = mbar_wait(bar(kBarPFull + x), np[x] & 1, abort_flag);
-              if (!ok) break;
-              ++np[x];
-              tc_fence_after();
-              issue_pv(x, v_base, i == 0);
-              if (next) {
-                // S(i+1) overwrites P(i) in place: the tensor pipe runs its operations in order
-                issue_qk(x, k_base);
-                if (i + 2 == w.n_tiles) umma_commit(bar(kBarQEmpty + x));
-              } else {
-                umma_commit(bar(kBarOFull + x));
-              }
-            }
+            const uint32_t k_stage = tk % KS, v_stage = tv % VS;
+            if (next) ok = mbar_wait(bar(kBarKFull + k_stage), (tk / KS) & 1, abort_flag);
+            if (ok) ok = mbar_wait(bar(kBarVFull + v_stage), (tv / VS) & 1, abort_flag);
+            if (ok) ok = chain(0, np0, ni0, i, w.n_tiles, k_stage, v_stage);
+            if (ok && w.has_b) ok = chain(1, np1, ni1, i, w.n_tiles, k_stage, v_stage);
             if (!ok) break;
-            umma_commit(bar(kBarVEmpty + tv % VS));
+            umma_commit(bar(kBarVEmpty + v_stage));
             ++tv;
             if (next) {
-              umma_commit(bar(kBarKEmpty + tk % KS));
+              umma_commit(bar(kBarKEmpty + k_stage));
               ++tk;
             }
           }
-          for (int x = 0; x < nx; ++x) ++ni[x];
+          ++ni0;
+          if (w.has_b) ++ni1;
         }
       }
       if (!ok) {
