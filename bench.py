@@ -109,6 +109,36 @@ def resolve_workload(name: str, probes_override=None) -> wl.Workload:
     return w
 
 
+def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 172e9) -> int:
+    """Layers assembled and attended per call: as many as fit beside the pool, the query-side
+    tensors and the outputs, at most 36 GB of assembled K + V."""
+    n_tok = float(wl.shot_lengths(w).sum())
+    pool_bytes = n_tok * w.bytes_per_token_layer * w.n_layers
+    q_bytes = (w.batch * w.n_layers * max(1, len(w.probes)) * w.t_q * (w.n_q_heads + 2 * w.n_kv_heads)
+               * w.head_dim * w.elem_size)
+    per_layer = float(w.batch) * ctx_cap * w.bytes_per_token_layer
+    budget = min(36e9, 0.5 * (device_bytes - pool_bytes - 3.0 * q_bytes))
+    return int(max(1, min(w.n_layers, budget // per_layer)))
+
+
+def planned_ctx_cap(ab, dpool, q_emb, w: wl.Workload) -> int:
+    """Capacity of the assembled cache: the longest planned context (selection + plan-only
+    call of the library), rounded up to the 128-token tile the attention kernel reads."""
+    dev = q_emb.device
+    sel = torch.empty((w.batch, w.k), dtype=torch.int32, device=dev)
+    off = torch.empty((w.batch, w.k + 1), dtype=torch.int64, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(max(256, ab.adapshot_select_workspace_bytes(dpool.c.n_shots, w.batch, w.k)),
+                     dtype=torch.uint8, device=dev)
+    model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
+    ab.adapshot_select(dpool, q_emb, w.k, sel, None, ws, st)
+    ab.adapshot_assemble_kv(model, dpool, sel, 0, 1, None, None, 0, off, st)
+    torch.cuda.synchronize()
+    if st.item() != 0:
+        raise SystemExit(f"device status {st.item()} while planning")
+    return int(-(-int(off[:, -1].max().item()) // 128) * 128)
+
+
 def algorithmic_counts(w: wl.Workload, ctx_off: np.ndarray, n_layers: int):
     """Algorithmic bytes / flops of one step from the plan (per the design doc's per-unit figures)."""
     L = ctx_off[:, -1].astype(np.float64)                         # longest probe per query
@@ -224,16 +254,16 @@ def run_ours(args, w: wl.Workload):
     n_pool_layers = min(w.n_layers, args.pool_layers) if args.pool_layers else w.n_layers
     pool = wl.make_pool(w, dev, n_layers=n_pool_layers)
     wq = w.scaled(seed=w.seed + 100 * rank) if rank else w
-    lpc = args.layers_per_call or w.n_layers
     so = torch.from_numpy(pool["shot_off"]).to(dev)
     k_pool, v_pool = pool["k"], pool["v"]
     if n_pool_layers < w.n_layers:
         raise SystemExit("layer aliasing is not implemented; the pool must hold every layer")
     dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
-    ctx_cap = args.ctx_cap or w.k * w.len_hi
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc)
     qs = wl.make_queries(wq, dev)
+    ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
+    lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap)
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
     del qs
@@ -248,7 +278,6 @@ def run_ours(args, w: wl.Workload):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- tighten the capacity to the planned context (set-up, not timed)
     step()
     torch.cuda.synchronize()
     if path.status.item() != 0:
