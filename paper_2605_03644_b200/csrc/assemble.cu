@@ -14,6 +14,7 @@ namespace {
 
 constexpr int kPlanThreads = 256;
 constexpr int kTile = 128;   // the attention kernel reads the cache in 128-token tiles
+constexpr int kRun = 4;      // consecutive destination tokens per warp
 
 // One CTA per query: lengths of the selected shots, block-wide exclusive scan.
 __global__ void __launch_bounds__(kPlanThreads)
@@ -137,15 +138,46 @@ gather_rope_kernel(const GatherArgs a) {
   uint4* kc = static_cast<uint4*>(a.k_ctx);
   uint4* vc = static_cast<uint4*>(a.v_ctx);
 
-  const long long units = (long long)a.B * a.ctx_cap;
-  for (long long u = warp_global; u < units; u += n_warps) {
-    const int b = (int)(u / a.ctx_cap);
-    const long long p = u % a.ctx_cap;
+  // A warp takes a run of kRun consecutive destination tokens of one query.  The plan lookup
+  // (which selected shot covers the position) is a dependent chain of global loads, so it is
+  // done once per run by the whole warp (a 32-ary search: two rounds of parallel probes of the
+  // offsets instead of log2(k) serial ones) and then walked forward token by token.
+  const long long runs_per_query = (a.ctx_cap + kRun - 1) / kRun;
+  const long long n_runs = (long long)a.B * runs_per_query;
+  for (long long run = warp_global; run < n_runs; run += n_warps) {
+    const int b = (int)(run / runs_per_query);
+    const long long p0 = (run % runs_per_query) * kRun;
     const long long* off = a.ctx_off + (long long)b * (a.k + 1);
     const long long L = off[a.k];
+    const long long pad_end = (L + kTile - 1) / kTile * kTile;
+    if (p0 >= pad_end) continue;
+    int lo = 0;
+    long long o = 0, o_next = 0, src0 = 0;
+    int s = -1;
+    if (p0 < L) {
+      // largest lo in [0, k) with off[lo] <= p0 (zero-length slots are skipped by the search)
+      int seg_lo = 0, seg_n = a.k;
+      while (seg_n > 1) {
+        const int stride = (seg_n + 31) / 32;
+        const int idx = seg_lo + lane * stride;
+        const bool le = idx < seg_lo + seg_n && off[idx] <= p0;
+        const int cnt = __popc(__ballot_sync(0xffffffffu, le));      // probes are ascending: a prefix is true
+        const int first = seg_lo + (cnt - 1) * stride;                // cnt >= 1: off[seg_lo] <= p0
+        seg_n = min(stride, seg_lo + seg_n - first);
+        seg_lo = first;
+      }
+      lo = seg_lo;
+      o = off[lo];
+      o_next = off[lo + 1];
+      s = a.sel_idx[(long long)b * a.k + lo];
+      if (s >= 0 && s < a.n_shots) src0 = a.shot_off[s];
+    }
+#pragma unroll 1
+    for (int tt = 0; tt < kRun; ++tt) {
+    const long long p = p0 + tt;
+    if (p >= a.ctx_cap) break;
     if (p >= L) {
       // zero the rest of the last 128-token tile so whole tiles can be read later
-      const long long pad_end = (L + kTile - 1) / kTile * kTile;
       if (p < pad_end) {
         for (int l = 0; l < a.n_layers_call; ++l) {
           const long long dst = ((long long)b * a.n_layers_call + l) * layer_stride_ctx + p * row_vecs;
@@ -157,16 +189,17 @@ gather_rope_kernel(const GatherArgs a) {
       }
       continue;
     }
-    // shot slot r with off[r] <= p < off[r+1] (zero-length slots are skipped by the search)
-    int lo = 0, hi = a.k;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (off[mid] <= p) lo = mid; else hi = mid;
+    if (p >= o_next) {               // next selected shot (skipping zero-length slots); warp-uniform
+      do {
+        ++lo;
+        o = o_next;
+        o_next = off[lo + 1];
+      } while (p >= o_next);
+      s = a.sel_idx[(long long)b * a.k + lo];
+      src0 = (s >= 0 && s < a.n_shots) ? a.shot_off[s] : 0;
     }
-    const long long o = off[lo];
-    const int s = a.sel_idx[(long long)b * a.k + lo];
     if (s < 0 || s >= a.n_shots) continue;           // reported by the plan kernel
-    const long long src_tok = a.shot_off[s] + (p - o);
+    const long long src_tok = src0 + (p - o);
     const double delta = a.k_pos_mode == 0 ? (double)p : (double)o;
 
     float sn[EPV], cs[EPV];
@@ -223,12 +256,13 @@ gather_rope_kernel(const GatherArgs a) {
         if (i + 96 < row_vecs) vc[dst + i + 96] = r3;
       }
     }
+    }
   }
 }
 
 template <typename T, int D>
 int launch_gather(const GatherArgs& a, cudaStream_t st) {
-  const long long units = (long long)a.B * a.ctx_cap;
+  const long long units = (long long)a.B * ((a.ctx_cap + kRun - 1) / kRun);
   const int warps_per_block = 8;
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
   const long long max_blocks = 148ll * 8 * 4;   // a few waves of resident CTAs, grid-stride beyond
