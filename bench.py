@@ -109,7 +109,7 @@ def resolve_workload(name: str, probes_override=None) -> wl.Workload:
     return w
 
 
-def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 172e9) -> int:
+def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e9) -> int:
     """Layers assembled and attended per call: as many as fit beside the pool, the query-side
     tensors and the outputs, at most 36 GB of assembled K + V."""
     n_tok = float(wl.shot_lengths(w).sum())
@@ -268,7 +268,8 @@ def run_ours(args, w: wl.Workload):
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
     del qs
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    launches_per_step = 2 + (1 if w.n_shots > 8192 else 0) + len(path.chunks) * (2 + 3) + 2
+    launches_per_step = 2 + (1 if w.n_shots > 8192 else 0) + (1 if path.overlap else 0) + \
+        len(path.chunks) * ((1 if path.overlap else 2) + 3) + 2
 
     def step():
         path.run(q_emb, qc, kqc, vqc, logits, args.tau)
@@ -433,7 +434,7 @@ def run_ours(args, w: wl.Workload):
             "config": {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
                        "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool["n_shots"]),
                        "pool_tokens": int(pool["pool_tokens"]), "ctx_tokens_per_step": counts["ctx_tokens"],
-                       "ctx_cap": ctx_cap, "layers_per_call": lpc, "l2": "flushed between steps (512 MiB write)",
+                       "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
                        "parallelism": "replicas" if world > 1 else "single"},
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

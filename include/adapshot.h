@@ -108,12 +108,17 @@ ADAPSHOT_API int adapshot_select(const adapshot_pool_t* pool, const float* q_emb
  *   Rot(x)_i = x_i cos - x_{i+d/2} sin, Rot(x)_{i+d/2} = x_{i+d/2} cos + x_i sin
  *   (Eq. 6, half-split rotate_half).  Angles are formed in fp64, the rotation in
  *   fp32, bf16 results are rounded to nearest-even.
- *   k_ctx, v_ctx : [B][nl][ctx_cap][Hkv][d]; both NULL => only ctx_off is written.
+ *   k_ctx, v_ctx : [B][nl][ctx_cap][Hkv][d]; both NULL => only ctx_off is written
+ *   (and, when ctx_cap > 0, the capacity is checked).
  *   Rows L .. min(roundup(L,128), ctx_cap)-1 of every (b, l) are zero-filled so
  *   that the attention kernel can read whole 128-token tiles.
  *   Device-detected: L > ctx_cap -> ADAPSHOT_ECAPACITY (tokens beyond the
  *   capacity are dropped); shot id out of range -> ADAPSHOT_EINDEX (the shot
- *   counts as length 0).  sel_idx need not come from adapshot_select.           */
+ *   counts as length 0).  sel_idx need not come from adapshot_select.
+ *   flags: 0, or ADAPSHOT_ASSEMBLE_KEEP_PLAN when ctx_off already holds the plan of
+ *   the same sel_idx (an earlier call): it is then read, not written, so calls for
+ *   further layer ranges may run on other streams while attention reads it.      */
+#define ADAPSHOT_ASSEMBLE_KEEP_PLAN 1u
 ADAPSHOT_API int adapshot_assemble_kv(const adapshot_model_t* model, const adapshot_pool_t* pool,
                          const int32_t* sel_idx, int32_t B, int32_t k,
                          int32_t layer_begin, int32_t layer_end,

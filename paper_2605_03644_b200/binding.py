@@ -22,6 +22,7 @@ lib = C.CDLL(_LIB_PATH)
 
 OK, EINVAL, ESHAPE, EALIGN, ECAPACITY, EUNSUPPORTED, ECUDA, EINDEX, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 F32, BF16 = 0, 1
+ASSEMBLE_KEEP_PLAN = 1
 
 EXPORTS = [
     "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",

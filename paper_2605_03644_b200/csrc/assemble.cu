@@ -109,8 +109,11 @@ struct GatherArgs {
 
 // D = head_dim.  A "pair unit" is the 16-byte vector j of the low half of one head
 // together with vector j of the high half (elements i and i + D/2 rotate together).
+// 128-thread CTAs of at most 88 registers: small enough to be co-resident with a persistent
+// attention CTA (which leaves about 11.7 K registers and 1.5 KB of shared memory per SM), so
+// that the gather of the next layer chunk can run under the attention of the current one.
 template <typename T, int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128, 6)
 gather_rope_kernel(const GatherArgs a) {
   constexpr int EPV = Vec16<T>::N;                 // elements per 16-byte vector
   constexpr int VPH = D / EPV;                     // vectors per head row
@@ -263,9 +266,9 @@ gather_rope_kernel(const GatherArgs a) {
 template <typename T, int D>
 int launch_gather(const GatherArgs& a, cudaStream_t st) {
   const long long units = (long long)a.B * ((a.ctx_cap + kRun - 1) / kRun);
-  const int warps_per_block = 8;
+  const int warps_per_block = 4;
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
-  const long long max_blocks = 148ll * 8 * 4;   // a few waves of resident CTAs, grid-stride beyond
+  const long long max_blocks = 148ll * 16 * 4;   // a few waves of resident CTAs, grid-stride beyond
   if (blocks > max_blocks) blocks = max_blocks;
   gather_rope_kernel<T, D><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
   return ads_launch_status();
@@ -279,9 +282,12 @@ extern "C" int adapshot_assemble_kv(const adapshot_model_t* model, const adapsho
                                     int64_t ctx_cap, int64_t* ctx_off, uint32_t flags,
                                     int32_t* status, void* stream) {
   if (model == nullptr || pool == nullptr || sel_idx == nullptr || ctx_off == nullptr) return ADAPSHOT_EINVAL;
-  if (B <= 0 || flags != 0 || pool->shot_off == nullptr || pool->n_shots <= 0) return ADAPSHOT_EINVAL;
+  if (B <= 0 || (flags & ~ADAPSHOT_ASSEMBLE_KEEP_PLAN) != 0 || pool->shot_off == nullptr || pool->n_shots <= 0)
+    return ADAPSHOT_EINVAL;
   if (k < 1 || k > pool->n_shots) return ADAPSHOT_ESHAPE;
   const bool plan_only = k_ctx == nullptr && v_ctx == nullptr;
+  const bool keep_plan = (flags & ADAPSHOT_ASSEMBLE_KEEP_PLAN) != 0;
+  if (plan_only && keep_plan) return ADAPSHOT_EINVAL;
   if (!plan_only && (k_ctx == nullptr || v_ctx == nullptr)) return ADAPSHOT_EINVAL;
   if (((uintptr_t)sel_idx & 3u) || ((uintptr_t)ctx_off & 7u)) return ADAPSHOT_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -299,10 +305,12 @@ extern "C" int adapshot_assemble_kv(const adapshot_model_t* model, const adapsho
       return ADAPSHOT_EALIGN;
   }
 
-  plan_offsets_kernel<<<B, kPlanThreads, 0, st>>>(
-      sel_idx, reinterpret_cast<const long long*>(pool->shot_off), pool->n_shots, k, ctx_cap, !plan_only,
-      reinterpret_cast<long long*>(ctx_off), status);
-  if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  if (!keep_plan) {
+    plan_offsets_kernel<<<B, kPlanThreads, 0, st>>>(
+        sel_idx, reinterpret_cast<const long long*>(pool->shot_off), pool->n_shots, k, ctx_cap, ctx_cap > 0,
+        reinterpret_cast<long long*>(ctx_off), status);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  }
   if (plan_only) return ADAPSHOT_OK;
 
   GatherArgs a;

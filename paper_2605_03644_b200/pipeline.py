@@ -3,8 +3,10 @@
 It owns the device buffers (assembled cache, offsets, workspaces, outputs) so a
 caller can run many queries without allocating; it does no arithmetic itself.
 Layers are processed in chunks of `layers_per_call`: assemble the chunk's cache,
-attend over it, reuse the buffer for the next chunk.  Query-side tensors come as one
-tensor per chunk, [B][layers in chunk][P][T_q][heads][d] (in a model, the queries of a
+attend over it, reuse the buffer for the next chunk.  `overlap=True` double-buffers the
+cache and enqueues the gather of chunk i+1 on a second stream; on B200 the persistent
+attention CTAs leave no room for a second resident kernel, so the two do not actually run
+together and the default is off.  Query-side tensors come as one tensor per chunk, [B][layers in chunk][P][T_q][heads][d] (in a model, the queries of a
 later layer do not exist before the earlier layers have run).
 """
 from __future__ import annotations
@@ -19,14 +21,13 @@ from . import binding as ab
 class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
-                 attn_flags: int = 0, device="cuda"):
+                 overlap: bool = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
         self.ctx_cap = int(ctx_cap)
         self.nl = model.n_layers
         self.lpc = self.nl if layers_per_call is None else int(layers_per_call)
-        self.attn_flags = attn_flags
         dt = torch.float32 if model.dtype == ab.F32 else torch.bfloat16
         hkv, hq, d = model.n_kv_heads, model.n_q_heads, model.head_dim
         u8 = dict(dtype=torch.uint8, device=device)
@@ -35,10 +36,11 @@ class ReusePath:
         self.sel_score = torch.empty((batch, k), dtype=torch.float32, device=device)
         self.ctx_off = torch.empty((batch, k + 1), dtype=torch.int64, device=device)
         self.chunks = [(lb, min(self.nl, lb + self.lpc)) for lb in range(0, self.nl, self.lpc)]
-        self._ctx_shape = lambda nl: (batch, nl, self.ctx_cap, hkv, d)
+        self.overlap = bool(overlap) and len(self.chunks) > 1
         n_ctx = batch * self.lpc * self.ctx_cap * hkv * d
-        self.k_buf = torch.empty(n_ctx, dtype=dt, device=device)
-        self.v_buf = torch.empty(n_ctx, dtype=dt, device=device)
+        n_buf = 2 if self.overlap else 1
+        self.k_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
+        self.v_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
         self.out = [torch.empty((batch, le - lb, self.P, t_q, hq, d), dtype=dt, device=device)
                     for lb, le in self.chunks]
         self.H = torch.empty((batch * self.P,), dtype=torch.float32, device=device)
@@ -47,35 +49,63 @@ class ReusePath:
         self.ws_attn = torch.empty(max(256, ab.adapshot_attn_workspace_bytes(model, batch, self.P, t_q, self.lpc,
                                                                               self.ctx_cap)), **u8)
         self.ws_entropy = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(batch * self.P, vocab)), **u8)
+        if self.overlap:
+            self.side = torch.cuda.Stream(device=device)
+            self.ev_plan = torch.cuda.Event()
+            self.ev_asm = [torch.cuda.Event() for _ in range(2)]
+            self.ev_attn = [torch.cuda.Event() for _ in range(2)]
 
     def select(self, q_emb: torch.Tensor):
         ab.adapshot_select(self.pool, q_emb, self.k, self.sel_idx, self.sel_score, self.ws_select, self.status)
 
-    def ctx_views(self, nl: int):
-        shape = self._ctx_shape(nl)
+    def plan(self):
+        """Destination offsets of the selected shots (and the capacity check)."""
+        ab.adapshot_assemble_kv(self.model, self.pool, self.sel_idx, 0, 1, None, None, self.ctx_cap,
+                                self.ctx_off, self.status)
+
+    def ctx_views(self, nl: int, buf: int = 0):
+        shape = (self.B, nl, self.ctx_cap, self.model.n_kv_heads, self.model.head_dim)
         n = shape[0] * shape[1] * shape[2] * shape[3] * shape[4]
-        return self.k_buf[:n].view(shape), self.v_buf[:n].view(shape)
+        return self.k_bufs[buf][:n].view(shape), self.v_bufs[buf][:n].view(shape)
 
-    def assemble(self, layer_begin: int, layer_end: int):
-        k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin)
+    def assemble(self, layer_begin: int, layer_end: int, buf: int = 0, keep_plan: bool = False):
+        k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin, buf)
         ab.adapshot_assemble_kv(self.model, self.pool, self.sel_idx, layer_begin, layer_end,
-                                k_ctx, v_ctx, self.ctx_cap, self.ctx_off, self.status)
+                                k_ctx, v_ctx, self.ctx_cap, self.ctx_off, self.status,
+                                flags=ab.ASSEMBLE_KEEP_PLAN if keep_plan else 0)
 
-    def attend(self, q, kq, vq, out, layer_begin: int, layer_end: int):
-        k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin)
+    def attend(self, q, kq, vq, out, layer_begin: int, layer_end: int, buf: int = 0):
+        k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin, buf)
         ab.adapshot_query_attn(self.model, k_ctx, v_ctx, self.ctx_cap, self.ctx_off,
                                self.k, self.probes, q, kq, vq, layer_begin, layer_end, out, None,
-                               self.ws_attn, self.status, flags=self.attn_flags)
+                               self.ws_attn, self.status)
 
     def entropy(self, logits: torch.Tensor, tau: float):
         ab.adapshot_entropy(logits, self.H, tau, self.P, self.first_ok, self.ws_entropy, self.status)
 
     def run(self, q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau: float = 0.65):
-        """One pass of the whole path; everything is enqueued on the current stream.
+        """One pass of the whole path; everything is enqueued on the current stream (the
+        gathers of a multi-chunk pass on the side stream, ordered by events).
         q_chunks[i] / kq_chunks[i] / vq_chunks[i] belong to layer chunk self.chunks[i]."""
         self.select(q_emb)
-        for i, (lb, le) in enumerate(self.chunks):
-            self.assemble(lb, le)
-            self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
+        if not self.overlap:
+            for i, (lb, le) in enumerate(self.chunks):
+                self.assemble(lb, le)
+                self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
+        else:
+            main = torch.cuda.current_stream()
+            self.plan()
+            self.ev_plan.record(main)
+            self.side.wait_event(self.ev_plan)
+            for i, (lb, le) in enumerate(self.chunks):
+                buf = i & 1
+                with torch.cuda.stream(self.side):
+                    if i >= 2:
+                        self.side.wait_event(self.ev_attn[buf])     # the buffer's last reader
+                    self.assemble(lb, le, buf, keep_plan=True)
+                    self.ev_asm[buf].record(self.side)
+                main.wait_event(self.ev_asm[buf])
+                self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le, buf)
+                self.ev_attn[buf].record(main)
         self.entropy(logits, tau)
         return self.out, self.H, self.first_ok

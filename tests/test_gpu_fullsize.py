@@ -11,6 +11,8 @@ the benchmark uses (pool resident on the device, capacity = planned context roun
   * entropy: every row, relative error 1e-4.
 Inputs are the seeded generators of paper_2605_03644_b200.workloads, made on the device; only
 the slices the oracle needs are copied to the host."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -48,6 +50,8 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0):
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
     dev = "cuda"
+    gc.collect()
+    torch.cuda.empty_cache()
     w = wl.CONFIGS[name]
     pool = wl.make_pool(w, dev)
     qs = wl.make_queries(w if w.probes else w.scaled(probes=(1,)), dev)
@@ -128,6 +132,7 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0):
     pad_end = min(-(-L // 128) * 128, ctx_cap)
     assert (k_ctx_d[b, l - lb, L:pad_end] == 0).all() and (v_ctx_d[b, l - lb, L:pad_end] == 0).all()
     del path, pool, qs, dpool, k_ctx_d, v_ctx_d
+    gc.collect()
     torch.cuda.empty_cache()
 
 
