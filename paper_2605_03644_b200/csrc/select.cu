@@ -1,6 +1,7 @@
 // Semantic shot selection (paper Sec. 4.1 ranking, Sec. 4.2 "rank in descending
 // order and select the top k"): cosine of the query embedding against every cached
-// shot embedding, then a block-wide top-k with ties broken by the lower shot id.
+// shot embedding, then the top k with ties broken by the lower shot id (by rank counting
+// for pools of up to 4096 shots, by chunked block-wide sorts beyond).
 //
 // The ranking must equal that of an fp64 evaluation of the same formula, so the
 // fp32 products (exact in fp64) are accumulated in fp64 and scores are compared in
@@ -161,6 +162,73 @@ topk_sort_kernel(const double* __restrict__ dots, const double* __restrict__ eno
   }
 }
 
+// Top-k by counting, for pools of up to kRankMaxN shots: the rank of shot i in the order
+// (score descending, id ascending) is the number of shots that precede it; every shot with
+// rank < k writes its id to position rank.  No sort and no serial phases: grid (N / 64, B),
+// 64 candidates per CTA, the comparison range split over four groups of 64 threads.
+// "key_j precedes key_i" = key_j < key_i, or equal keys and j < i, = key_j < key_i + (j < i).
+constexpr int kRankMaxN = 4096;
+constexpr int kRankThreads = 256, kRankCand = 64, kRankTile = 2048;
+
+__global__ void __launch_bounds__(kRankThreads)
+rank_topk_kernel(const double* __restrict__ dots, const double* __restrict__ enorm,
+                 const float* __restrict__ q_emb, int E, int N, int k,
+                 int32_t* __restrict__ final_idx, float* __restrict__ final_score) {
+  __shared__ unsigned long long keys[kRankTile];
+  __shared__ double red[kRankThreads / 32];
+  __shared__ double qnorm_sh;
+  __shared__ int part_cnt[kRankThreads];
+  const int b = blockIdx.y;
+  const int tid = threadIdx.x;
+  {
+    const float* q = q_emb + (long long)b * E;
+    double acc = 0.0;
+    for (int i = tid; i < E; i += kRankThreads) acc += (double)q[i] * q[i];
+    acc = warp_sum(acc);
+    if ((tid & 31) == 0) red[tid >> 5] = acc;
+    __syncthreads();
+    if (tid < 32) {
+      double v = tid < kRankThreads / 32 ? red[tid] : 0.0;
+      v = warp_sum(v);
+      if (tid == 0) qnorm_sh = sqrt(v);
+    }
+    __syncthreads();
+  }
+  const double qn = qnorm_sh;
+  auto key_of = [&](int j) -> unsigned long long {
+    const double den = qn * enorm[j];
+    const double sc = den > 0.0 ? dots[(long long)b * N + j] / den : 0.0;
+    return desc_key(sc);
+  };
+  const int i = blockIdx.x * kRankCand + (tid & (kRankCand - 1));
+  const int part = tid / kRankCand;                       // which quarter of every tile this thread scans
+  const unsigned long long ki = i < N ? key_of(i) : ~0ull;
+  const unsigned long long ki_le = ki == ~0ull ? ki : ki + 1;   // threshold for j < i (equal keys precede)
+  int cnt = 0;
+  for (int tile0 = 0; tile0 < N; tile0 += kRankTile) {
+    const int n_t = min(kRankTile, N - tile0);
+    for (int t = tid; t < n_t; t += kRankThreads) keys[t] = key_of(tile0 + t);
+    __syncthreads();
+    const int per = kRankTile / (kRankThreads / kRankCand);
+    const int j0 = part * per, j1 = min(n_t, j0 + per);
+    const int split = max(j0, min(j1, i - tile0));        // [j0, split): j < i;  [split, j1): j >= i
+    for (int j = j0; j < split; ++j) cnt += keys[j] < ki_le ? 1 : 0;
+    for (int j = split; j < j1; ++j) cnt += keys[j] < ki ? 1 : 0;
+    __syncthreads();
+  }
+  part_cnt[tid] = cnt;
+  __syncthreads();
+  if (part == 0 && i < N) {
+    int rank = 0;
+#pragma unroll
+    for (int q4 = 0; q4 < kRankThreads / kRankCand; ++q4) rank += part_cnt[q4 * kRankCand + tid];
+    if (rank < k) {
+      final_idx[(long long)b * k + rank] = i;
+      if (final_score != nullptr) final_score[(long long)b * k + rank] = (float)key_score(ki);
+    }
+  }
+}
+
 size_t sel_cand_entries(int n_shots, int k) {
   if (n_shots <= kSortCap) return 0;
   size_t chunks = ((size_t)n_shots + kSortCap - 1) / kSortCap;
@@ -187,7 +255,7 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
   if (pool->emb == nullptr || pool->n_shots <= 0 || pool->emb_dim <= 0 || B <= 0) return ADAPSHOT_EINVAL;
   const int N = pool->n_shots, E = pool->emb_dim;
   if (k < 1 || k > N) return ADAPSHOT_ESHAPE;
-  if (N > kSortCap && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
+  if (N > kRankMaxN && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
   if (!ads_aligned16(pool->emb) || !ads_aligned16(q_emb) || !ads_aligned16(ws)) return ADAPSHOT_EALIGN;
   if (ws_bytes < adapshot_select_workspace_bytes(N, B, k)) return ADAPSHOT_ECAPACITY;
 
@@ -211,6 +279,12 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
   cosine_dots_kernel<<<(N + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
       pool->emb, q_emb, N, E, B, dots, enorm);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+
+  if (N <= kRankMaxN) {
+    dim3 grid((N + kRankCand - 1) / kRankCand, B);
+    rank_topk_kernel<<<grid, kRankThreads, 0, st>>>(dots, enorm, q_emb, E, N, k, sel_idx, sel_score);
+    return ads_launch_status();
+  }
 
   const size_t smem = (size_t)kSortCap * (8 + 4);
   static bool attr_set = false;   // same value every time: a benign race
