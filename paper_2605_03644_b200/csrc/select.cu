@@ -255,7 +255,7 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
   if (pool->emb == nullptr || pool->n_shots <= 0 || pool->emb_dim <= 0 || B <= 0) return ADAPSHOT_EINVAL;
   const int N = pool->n_shots, E = pool->emb_dim;
   if (k < 1 || k > N) return ADAPSHOT_ESHAPE;
-  if (N > kRankMaxN && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
+  if (N > kSortCap && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
   if (!ads_aligned16(pool->emb) || !ads_aligned16(q_emb) || !ads_aligned16(ws)) return ADAPSHOT_EALIGN;
   if (ws_bytes < adapshot_select_workspace_bytes(N, B, k)) return ADAPSHOT_ECAPACITY;
 
