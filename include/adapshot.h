@@ -153,6 +153,25 @@ ADAPSHOT_API int adapshot_query_attn(const adapshot_model_t* model,
                         void* out, float* lse, uint32_t flags,
                         void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
+/* ---- Steps 2 + 3 fused: the same attention, but the context K/V tiles are read from
+ * the pool (through sel_idx / ctx_off) and K is re-encoded (Eq. 7) tile by tile in
+ * shared memory on its way to the tensor cores, so that no assembled cache is written
+ * to or read from HBM.  Results equal adapshot_assemble_kv + adapshot_query_attn up to
+ * the rounding of the rotary table (fp32 (cos, sin) from fp64 angles, neighbouring rows
+ * by one fp32 complex multiplication; K' rounded once to bf16 as in the materialised
+ * path).  ctx_off: the plan written by adapshot_assemble_kv (plan-only call is enough)
+ * for the same sel_idx; ctx_cap: an upper bound of every L (sizes the workspace: a row
+ * map of B * ctx_cap int32 and a table of ctx_cap * d * 4 bytes).  Needs
+ * model->k_pos_mode == 0, pool_tokens < 2^31.  Other arguments as above.             */
+ADAPSHOT_API size_t adapshot_attn_fused_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
+                                           int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap);
+ADAPSHOT_API int adapshot_query_attn_fused(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                              const int32_t* sel_idx, const int64_t* ctx_off, int64_t ctx_cap,
+                              int32_t B, int32_t k, const int32_t* probe_nshots, int32_t P,
+                              const void* q, const void* kq, const void* vq, int32_t Tq,
+                              int32_t layer_begin, int32_t layer_end, void* out, float* lse,
+                              uint32_t flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
 /* ---- Step 4: confidence probe (Eq. 2 over the whole vocabulary, natural log)
  * and the threshold rule that follows it.
  *   H[r] = -sum_v p_v ln p_v, p = softmax(logits[r][0..V))          (fp32 out)

@@ -27,6 +27,7 @@ ASSEMBLE_KEEP_PLAN = 1
 EXPORTS = [
     "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
+    "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_static",
     "adapshot_strerror", "adapshot_version",
 ]
@@ -67,6 +68,13 @@ _attn_ws = _sig("adapshot_attn_workspace_bytes", _sz, [C.POINTER(ModelT), _i32, 
 _attn = _sig("adapshot_query_attn", C.c_int,
              [C.POINTER(ModelT), _vp, _vp, _i64, _vp, _i32, _i32, C.POINTER(_i32), _i32,
               _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+
+
+_attn_fused_ws = _sig("adapshot_attn_fused_workspace_bytes", _sz,
+                      [C.POINTER(ModelT), _i32, _i32, _i32, _i32, _i64])
+_attn_fused = _sig("adapshot_query_attn_fused", C.c_int,
+                   [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _vp, _i64, _i32, _i32, C.POINTER(_i32), _i32,
+                    _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
 
 
 class AdapshotError(RuntimeError):
@@ -156,6 +164,25 @@ def adapshot_query_attn(model: ModelT, k_ctx: torch.Tensor, v_ctx: torch.Tensor,
     _check(_attn(C.byref(model), _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), B, k, arr, P,
                  _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
                  flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_attn_fused_workspace_bytes(model: ModelT, B: int, P: int, Tq: int, n_layers_in_call: int,
+                                        ctx_cap: int) -> int:
+    return _attn_fused_ws(C.byref(model), B, P, Tq, n_layers_in_call, ctx_cap)
+
+
+def adapshot_query_attn_fused(model: ModelT, pool: Pool, sel_idx: torch.Tensor, ctx_off: torch.Tensor,
+                              ctx_cap: int, probe_nshots: Sequence[int], q: torch.Tensor, kq: torch.Tensor,
+                              vq: torch.Tensor, layer_begin: int, layer_end: int, out: torch.Tensor,
+                              lse: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor,
+                              flags: int = 0):
+    B, k = sel_idx.shape
+    P = len(probe_nshots)
+    Tq = q.shape[3]
+    arr = (_i32 * P)(*[int(x) for x in probe_nshots])
+    _check(_attn_fused(C.byref(model), C.byref(pool.c), _ptr(sel_idx), _ptr(ctx_off), ctx_cap, B, k, arr, P,
+                       _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
+                       flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
 
 
 def adapshot_entropy_workspace_bytes(R: int, V: int) -> int:

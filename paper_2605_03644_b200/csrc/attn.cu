@@ -35,6 +35,8 @@ constexpr int kMaxGang = 8;          // CTAs that share one range of K/V tiles
 constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
 constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
+constexpr int kFusedThreads = 384;   // fused variant: warps 2-3 load and rotate K/V, softmax on warps 4-11
+constexpr int kLoaders = 64;         // threads of the two loader warps
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by 2^8
 constexpr float kNegSentinel = -1.0e30f;
@@ -63,6 +65,16 @@ struct AttnParams {
   int B, P, Tq, Hq, Hkv, G, nl;
   int n_mt, n_mp, gang, n_gangs;
   float scale_log2;           // softmax_scale * log2(e)
+  // fused variant only: K/V tiles come from the pool (and from the probe's own rotated keys)
+  const __nv_bfloat16* k_pool;   // [n_layers][pool_tokens][Hkv][D]
+  const __nv_bfloat16* v_pool;
+  const __nv_bfloat16* kq_rot;   // [B*nl*P][Tq][Hkv][D], rotated by the prep kernel
+  const __nv_bfloat16* vq;
+  const int* row_map;            // [B][ctx_cap]: pool token of every context position, -1 beyond L
+  const float2* rope_tab;        // [ctx_cap rounded up to 128][D/2]: (cos, sin) of position * theta_i
+  long long pool_tokens, ctx_cap;
+  int layer_begin;
+  double rope_base_f;
 };
 
 struct PrepParams {
@@ -182,6 +194,52 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   }
 }
 
+// Fused variant, once per call: the pool token behind every context position of every query
+// (the gather's plan lookup, stored instead of applied) and the rotary table of the context
+// positions, (cos, sin)(p * theta_i) from fp64 angles.
+struct FusedPlanParams {
+  const long long* ctx_off;   // [B][k+1]
+  const int32_t* sel_idx;     // [B][k]
+  const long long* shot_off;  // [n_shots+1]
+  int* row_map;               // [B][ctx_cap]
+  float2* rope_tab;           // [tab_rows][D/2]
+  long long ctx_cap, tab_rows;
+  int B, k, n_shots, half_d;
+  double rope_base;
+};
+
+__global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanParams p) {
+  const long long n_map = (long long)p.B * p.ctx_cap;
+  const long long n_tab = p.tab_rows * p.half_d;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < n_map + n_tab; u += stride) {
+    if (u < n_map) {
+      const int b = (int)(u / p.ctx_cap);
+      const long long pos = u % p.ctx_cap;
+      const long long* off = p.ctx_off + (long long)b * (p.k + 1);
+      int row = -1;
+      if (pos < off[p.k]) {
+        int lo = 0, hi = p.k;          // shot slot with off[lo] <= pos < off[lo+1]
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (off[mid] <= pos) lo = mid; else hi = mid;
+        }
+        const int s = p.sel_idx[(long long)b * p.k + lo];
+        if (s >= 0 && s < p.n_shots) row = (int)(p.shot_off[s] + (pos - off[lo]));
+      }
+      p.row_map[u] = row;
+    } else {
+      const long long v = u - n_map;
+      const long long pos = v / p.half_d;
+      const int i = (int)(v % p.half_d);
+      const double theta = pow(p.rope_base, -(double)i / (double)p.half_d);
+      float sn, cs;
+      rope_sincos((double)pos, theta, &sn, &cs);
+      p.rope_tab[v] = make_float2(cs, sn);
+    }
+  }
+}
+
 // Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
 template <int D>
@@ -278,8 +336,11 @@ __device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, 
 
 // TMEM: S/P of M tile A at columns 0..127, of M tile B at 128..255 (P, as packed bf16,
 // overwrites the S tile it was computed from); O accumulators at 256 and 384.
-template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+// FUSED: the context K/V tiles are read from the pool through the row map (per-thread async
+// copies into the swizzled tile layout) and K is rotated in shared memory by two loader warps,
+// so that no re-encoded cache is ever written to HBM; TMA then only brings Q.
+template <int D, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? kFusedThreads : kAttnThreads, 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
                  const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
@@ -315,9 +376,9 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       mbar_init(bar(kBarOEmpty + i), 128);
     }
     for (int i = 0; i < 3; ++i) {
-      mbar_init(bar(kBarKFull + i), 1);
+      mbar_init(bar(kBarKFull + i), FUSED ? kLoaders : 1);
       mbar_init(bar(kBarKEmpty + i), 1);
-      mbar_init(bar(kBarVFull + i), 1);
+      mbar_init(bar(kBarVFull + i), FUSED ? kLoaders : 1);
       mbar_init(bar(kBarVEmpty + i), 1);
     }
     mbar_init(bar(kBarDrain), 1);
@@ -362,7 +423,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                           (2 * mp + x) * kTileM, w.outer_q);
             ++nq[x];
           }
-          for (int i = 0; i < w.n_tiles && ok; ++i) {
+          for (int i = 0; i < (FUSED ? 0 : w.n_tiles) && ok; ++i) {
             const bool own = i >= w.n_ctx;
             const CUtensorMap* mk = own ? &tm_kown : &tm_kctx;
             const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
@@ -389,12 +450,14 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           }
         }
       }
-      if (!ok) {
+      if (!ok && !FUSED) {
         // gave up: let the copies already in flight land before the CTA retires
         for (uint32_t t = tk > (uint32_t)KS ? tk - KS : 0; t < tk; ++t)
           mbar_wait(bar(kBarKFull + t % KS), (t / KS) & 1, abort_flag + 1);
         for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
           mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
+      }
+      if (!ok) {
         for (int x = 0; x < 2; ++x)
           if (nq[x] > 0) mbar_wait(bar(kBarQFull + x), (nq[x] - 1) & 1, abort_flag + 1);
       }
@@ -498,9 +561,148 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
     __syncwarp();
+  } else if (FUSED && warp < 4) {
+    // ------------------------------------------- loader: K/V tiles straight from the pool
+    // A thread owns the same rotary pairs of every tile: pair c = lt + 64 u is row c / PPR,
+    // 16-byte chunk jj = c % PPR of the low half and chunk jj + PPR of the high half, so its
+    // eight frequencies never change and consecutive pairs are kRowStep positions apart: the
+    // (cos, sin) of the first row come from the table, the others by one complex
+    // multiplication with (cos, sin)(kRowStep * theta).  Copies are per-thread async copies
+    // (no registers, zero fill for rows beyond the context), written in the 128-byte swizzle
+    // the UMMA descriptors expect; K is rotated in place by the thread that copied it.
+    constexpr int PPR = D / 16;
+    constexpr int kRowStep = kLoaders / PPR;
+    constexpr int PAIRS = kTileN / kRowStep;
+    const int lt = threadIdx.x - 64;
+    const int jj = lt % PPR, row0 = lt / PPR;
+    uint32_t dst_off[2];                              // tile offsets of row 0's two chunks, before the row term
+#pragma unroll
+    for (int h = 0; h < 2; ++h) dst_off[h] = ((jj + h * PPR) / 8) * 16384u;
+    float2 step[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const double theta = pow((double)p.rope_base_f, -(double)(jj * 8 + e) / (double)(D / 2));
+      float sn, cs;
+      rope_sincos((double)kRowStep, theta, &sn, &cs);
+      step[e] = make_float2(cs, sn);
+    }
+    uint32_t tk = 0, tv = 0;
+    bool ok = true;
+    Walker wk = wk0;
+    Piece pc;
+    auto chunk_addr = [&](int row, int h) -> uint32_t {
+      const int j = (jj + h * PPR) & 7;
+      return dst_off[h] + row * 128u + ((j ^ (row & 7)) << 4);
+    };
+    auto issue = [&](const Item& w, int i, uint32_t sk, uint32_t sv) {
+      const bool own = i >= w.n_ctx;
+      const uint32_t k_base = base + SM::kOffK + sk * kTileBytes, v_base = base + SM::kOffV + sv * kTileBytes;
+      long long src[PAIRS];                            // element offset of the row's head, -1: zero fill
+#pragma unroll
+      for (int u = 0; u < PAIRS; ++u) {
+        const int row = row0 + u * kRowStep;
+        if (!own) {
+          const long long pos = (long long)(w.ctx_begin + i) * kTileN + row;
+          const int r = pos < p.ctx_cap ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
+          src[u] = r < 0 ? -1 : (((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g) * D;
+        } else {
+          const int t = (w.own_begin + i - w.n_ctx) * kTileN + row;
+          src[u] = t >= p.Tq ? -1 : (((long long)w.outer_own * p.Tq + t) * p.Hkv + w.g) * D;
+        }
+      }
+      const __nv_bfloat16* kb = own ? p.kq_rot : p.k_pool;
+      const __nv_bfloat16* vb = own ? p.vq : p.v_pool;
+#pragma unroll
+      for (int u = 0; u < PAIRS; ++u) {
+        const int row = row0 + u * kRowStep;
+        const uint32_t n = src[u] < 0 ? 0u : 16u;
+        const __nv_bfloat16* g = kb + (src[u] < 0 ? 0 : src[u]) + jj * 8;
+        cp_async16(k_base + chunk_addr(row, 0), g, n);
+        cp_async16(k_base + chunk_addr(row, 1), g + D / 2, n);
+      }
+      cp_async_commit();
+#pragma unroll
+      for (int u = 0; u < PAIRS; ++u) {
+        const int row = row0 + u * kRowStep;
+        const uint32_t n = src[u] < 0 ? 0u : 16u;
+        const __nv_bfloat16* g = vb + (src[u] < 0 ? 0 : src[u]) + jj * 8;
+        cp_async16(v_base + chunk_addr(row, 0), g, n);
+        cp_async16(v_base + chunk_addr(row, 1), g + D / 2, n);
+      }
+      cp_async_commit();
+    };
+    auto rotate = [&](const Item& w, int i, uint32_t sk) {
+      unsigned char* kt = base_ptr + SM::kOffK + sk * kTileBytes;
+      const long long pos0 = (long long)(w.ctx_begin + i) * kTileN + row0;
+      float2 cur[8];
+      const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + pos0 * (D / 2) + jj * 8);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 t4 = tab[e];
+        cur[2 * e] = make_float2(t4.x, t4.y);
+        cur[2 * e + 1] = make_float2(t4.z, t4.w);
+      }
+#pragma unroll
+      for (int u = 0; u < PAIRS; ++u) {
+        const int row = row0 + u * kRowStep;
+        uint4* lo = reinterpret_cast<uint4*>(kt + chunk_addr(row, 0));
+        uint4* hi = reinterpret_cast<uint4*>(kt + chunk_addr(row, 1));
+        float x[8], y[8], xr[8], yr[8];
+        bf16x8_unpack(*lo, x);
+        bf16x8_unpack(*hi, y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          xr[e] = x[e] * cur[e].x - y[e] * cur[e].y;
+          yr[e] = y[e] * cur[e].x + x[e] * cur[e].y;
+        }
+        *lo = bf16x8_pack(xr);
+        *hi = bf16x8_pack(yr);
+        if (u + 1 < PAIRS) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float c = cur[e].x * step[e].x - cur[e].y * step[e].y;
+            const float sn = cur[e].y * step[e].x + cur[e].x * step[e].y;
+            cur[e] = make_float2(c, sn);
+          }
+        }
+      }
+    };
+    while (ok && next_piece(sc, n_pairs, wk, pc)) {
+      for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
+        Item w;
+        make_item(p, pc, gang_id, mp, w);
+        if (w.n_tiles == 0) continue;
+        ok = mbar_wait(bar(kBarKEmpty + tk % KS), ((tk / KS) & 1) ^ 1, abort_flag) &&
+             mbar_wait(bar(kBarVEmpty + tv % VS), ((tv / VS) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        issue(w, 0, tk % KS, tv % VS);
+        for (int i = 0; i < w.n_tiles; ++i) {
+          const uint32_t sk = tk % KS, sv = tv % VS;
+          const bool next = i + 1 < w.n_tiles;
+          if (next) {
+            ok = mbar_wait(bar(kBarKEmpty + (tk + 1) % KS), (((tk + 1) / KS) & 1) ^ 1, abort_flag) &&
+                 mbar_wait(bar(kBarVEmpty + (tv + 1) % VS), (((tv + 1) / VS) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            issue(w, i + 1, (tk + 1) % KS, (tv + 1) % VS);
+            cp_async_wait<3>();                         // K of tile i has landed
+          } else {
+            cp_async_wait<1>();
+          }
+          if (i < w.n_ctx) rotate(w, i, sk);
+          fence_proxy_async_smem();
+          mbar_arrive(bar(kBarKFull + sk));
+          if (next) cp_async_wait<2>(); else cp_async_wait<0>();   // V of tile i
+          fence_proxy_async_smem();
+          mbar_arrive(bar(kBarVFull + sv));
+          ++tk;
+          ++tv;
+        }
+      }
+    }
+    cp_async_wait<0>();
   } else {
     // ---------------------------------------------------- softmax + read-out of O
-    const int x = (warp - 2) >> 2;                 // 0: M tile A, 1: M tile B
+    const int x = (warp - (FUSED ? 4 : 2)) >> 2;   // 0: M tile A, 1: M tile B
     const int quarter = warp & 3;                  // TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;             // row of the M tile
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
@@ -758,12 +960,20 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 
 struct AttnPlan {
   int n_mt, n_mp, gang;
-  size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, total;
+  size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, off_rowmap, off_tab, total;
+  long long tab_rows;
+};
+
+// What the fused variant reads instead of an assembled cache.
+struct FusedSrc {
+  const adapshot_pool_t* pool;
+  const int32_t* sel_idx;
+  int layer_begin;
 };
 
 // The gang (CTAs that walk the same K/V tiles, one M pair each per round) is the number of
 // M pairs when that is at most kMaxGang, else the M pairs are dealt out in rounds.
-AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl) {
+AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, long long fused_ctx_cap = 0) {
   AttnPlan pl;
   const int G = model->n_q_heads / model->n_kv_heads;
   const int D = model->head_dim;
@@ -778,6 +988,13 @@ AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl) 
   pl.off_sched = off; off += ads_round_up(sizeof(Sched), 256);
   pl.off_opart = off; off += ads_round_up(slots * 2 * kTileM * D * 4, 256);
   pl.off_ml = off;    off += ads_round_up(slots * 2 * kTileM * 2 * 4, 256);
+  pl.off_rowmap = pl.off_tab = off;
+  pl.tab_rows = 0;
+  if (fused_ctx_cap > 0) {
+    pl.tab_rows = (fused_ctx_cap + kTileN - 1) / kTileN * kTileN;
+    pl.off_rowmap = off; off += ads_round_up((size_t)B * fused_ctx_cap * 4, 256);
+    pl.off_tab = off;    off += ads_round_up((size_t)pl.tab_rows * (D / 2) * 8, 256);
+  }
   pl.total = off;
   return pl;
 }
@@ -791,7 +1008,7 @@ template <int D>
 int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx, int64_t ctx_cap,
                 const int64_t* ctx_off, int B, int k, const int32_t* probe_nshots, int P, const void* q,
                 const void* kq, const void* vq, int Tq, int nl, void* out, float* lse, const AttnPlan& pl,
-                void* ws, int32_t* status, cudaStream_t st) {
+                void* ws, int32_t* status, cudaStream_t st, const FusedSrc* fused = nullptr) {
   const int Hq = model->n_q_heads, Hkv = model->n_kv_heads, G = Hq / Hkv;
   unsigned char* wsb = static_cast<unsigned char*>(ws);
   __nv_bfloat16* q_rot = reinterpret_cast<__nv_bfloat16*>(wsb + pl.off_qrot);
@@ -821,8 +1038,13 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)ctx_cap, (uint64_t)B * nl};
     const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, (uint64_t)ctx_cap * Hkv * D * 2};
     const uint32_t box[4] = {64, 1, (uint32_t)kTileN, 1};
-    if (!make_map(&tm_kctx, k_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
-    if (!make_map(&tm_vctx, v_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    if (fused != nullptr) {
+      tm_kctx = tm_q;                  // never used: the loader warps read the pool
+      tm_vctx = tm_q;
+    } else {
+      if (!make_map(&tm_kctx, k_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+      if (!make_map(&tm_vctx, v_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    }
   }
   {
     const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)Tq, (uint64_t)B * nl * P};
@@ -830,6 +1052,25 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     const uint32_t box[4] = {64, 1, (uint32_t)kTileN, 1};
     if (!make_map(&tm_kown, kq_rot, 4, dims, str, box)) return ADAPSHOT_ECUDA;
     if (!make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+  }
+
+  // ---- fused variant: row map and rotary table
+  int* row_map = reinterpret_cast<int*>(wsb + pl.off_rowmap);
+  float2* rope_tab = reinterpret_cast<float2*>(wsb + pl.off_tab);
+  if (fused != nullptr) {
+    FusedPlanParams fp;
+    fp.ctx_off = reinterpret_cast<const long long*>(ctx_off);
+    fp.sel_idx = fused->sel_idx;
+    fp.shot_off = reinterpret_cast<const long long*>(fused->pool->shot_off);
+    fp.row_map = row_map; fp.rope_tab = rope_tab;
+    fp.ctx_cap = ctx_cap; fp.tab_rows = pl.tab_rows;
+    fp.B = B; fp.k = k; fp.n_shots = fused->pool->n_shots; fp.half_d = D / 2;
+    fp.rope_base = model->rope_base;
+    const long long work = (long long)B * ctx_cap + pl.tab_rows * (D / 2);
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    attn_fused_plan_kernel<<<(unsigned)blocks, 256, 0, st>>>(fp);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   }
 
   // ---- rotate Q and the probe's own K, write the schedule
@@ -845,7 +1086,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   // ---- main kernel
-  AttnParams ap;
+  AttnParams ap = {};
   ap.sched = sched; ap.o_part = o_part; ap.ml_part = ml_part;
   ap.out = static_cast<__nv_bfloat16*>(out); ap.lse = lse; ap.status = status;
   ap.B = B; ap.P = P; ap.Tq = Tq; ap.Hq = Hq; ap.Hkv = Hkv; ap.G = G; ap.nl = nl;
@@ -853,13 +1094,31 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
   const int smem = (int)AttnSmem<128>::kTotal;     // same request for D = 64: one CTA per SM
-  static bool attr_done[2] = {false, false};
-  if (!attr_done[D == 128]) {
-    ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_done[D == 128] = true;
+  static bool attr_done[2][2] = {{false, false}, {false, false}};
+  if (fused == nullptr) {
+    if (!attr_done[0][D == 128]) {
+      ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          smem));
+      attr_done[0][D == 128] = true;
+    }
+    attn_main_kernel<D, false><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(
+        tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+  } else {
+    ap.k_pool = static_cast<const __nv_bfloat16*>(fused->pool->k);
+    ap.v_pool = static_cast<const __nv_bfloat16*>(fused->pool->v);
+    ap.kq_rot = kq_rot;
+    ap.vq = static_cast<const __nv_bfloat16*>(vq);
+    ap.row_map = row_map; ap.rope_tab = rope_tab;
+    ap.pool_tokens = fused->pool->pool_tokens; ap.ctx_cap = ctx_cap;
+    ap.layer_begin = fused->layer_begin; ap.rope_base_f = model->rope_base;
+    if (!attr_done[1][D == 128]) {
+      ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          smem));
+      attr_done[1][D == 128] = true;
+    }
+    attn_main_kernel<D, true><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
+        tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   }
-  attn_main_kernel<D><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(tm_q, tm_kctx, tm_vctx, tm_kown,
-                                                                               tm_vown, ap);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   // ---- merge the units that a range boundary cut
@@ -914,4 +1173,52 @@ extern "C" int adapshot_query_attn(const adapshot_model_t* model, const void* k_
                             lse, pl, ws, status, st);
   return launch_attn<64>(model, k_ctx, v_ctx, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
                          lse, pl, ws, status, st);
+}
+
+extern "C" size_t adapshot_attn_fused_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
+                                                      int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap) {
+  if (model == nullptr || !attn_shape_ok(model) || B <= 0 || P <= 0 || Tq <= 0 || n_layers_in_call <= 0 ||
+      ctx_cap <= 0)
+    return 0;
+  return make_plan(model, B, P, Tq, n_layers_in_call, ctx_cap).total;
+}
+
+extern "C" int adapshot_query_attn_fused(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                                         const int32_t* sel_idx, const int64_t* ctx_off, int64_t ctx_cap,
+                                         int32_t B, int32_t k, const int32_t* probe_nshots, int32_t P,
+                                         const void* q, const void* kq, const void* vq, int32_t Tq,
+                                         int32_t layer_begin, int32_t layer_end, void* out, float* lse,
+                                         uint32_t flags, void* ws, size_t ws_bytes, int32_t* status,
+                                         void* stream) {
+  if (model == nullptr || pool == nullptr || sel_idx == nullptr || ctx_off == nullptr || probe_nshots == nullptr ||
+      q == nullptr || kq == nullptr || vq == nullptr || out == nullptr || ws == nullptr)
+    return ADAPSHOT_EINVAL;
+  if (pool->k == nullptr || pool->v == nullptr || pool->shot_off == nullptr || pool->n_shots <= 0 ||
+      pool->pool_tokens <= 0)
+    return ADAPSHOT_EINVAL;
+  if (B <= 0 || k <= 0 || Tq <= 0 || ctx_cap <= 0 || flags != 0) return ADAPSHOT_EINVAL;
+  if (model->dtype != ADAPSHOT_BF16 || model->k_pos_mode != 0) return ADAPSHOT_EUNSUPPORTED;
+  if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
+  if (!(model->rope_base > 1.0)) return ADAPSHOT_EINVAL;
+  if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
+  if (P < 1 || P > kMaxProbes || (long long)P * B > kMaxPairs || k > pool->n_shots) return ADAPSHOT_ESHAPE;
+  for (int i = 0; i < P; ++i) {
+    if (probe_nshots[i] < 1 || probe_nshots[i] > k) return ADAPSHOT_ESHAPE;
+    if (i > 0 && probe_nshots[i] <= probe_nshots[i - 1]) return ADAPSHOT_ESHAPE;
+  }
+  if (!ads_aligned16(pool->k) || !ads_aligned16(pool->v) || !ads_aligned16(q) || !ads_aligned16(kq) ||
+      !ads_aligned16(vq) || !ads_aligned16(out) || ((uintptr_t)ws & 255u) || ((uintptr_t)sel_idx & 3u))
+    return ADAPSHOT_EALIGN;
+  if (ctx_cap > (1ll << 31) - 256 || pool->pool_tokens > (1ll << 31) - 1) return ADAPSHOT_ESHAPE;
+  const int nl = layer_end - layer_begin;
+  const AttnPlan pl = make_plan(model, B, P, Tq, nl, ctx_cap);
+  if (ws_bytes < pl.total) return ADAPSHOT_ECAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FusedSrc src;
+  src.pool = pool; src.sel_idx = sel_idx; src.layer_begin = layer_begin;
+  if (model->head_dim == 128)
+    return launch_attn<128>(model, nullptr, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl,
+                            out, lse, pl, ws, status, st, &src);
+  return launch_attn<64>(model, nullptr, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
+                         lse, pl, ws, status, st, &src);
 }

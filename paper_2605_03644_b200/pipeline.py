@@ -3,7 +3,8 @@
 It owns the device buffers (assembled cache, offsets, workspaces, outputs) so a
 caller can run many queries without allocating; it does no arithmetic itself.
 Layers are processed in chunks of `layers_per_call`: assemble the chunk's cache,
-attend over it, reuse the buffer for the next chunk.  `overlap=True` double-buffers the
+attend over it, reuse the buffer for the next chunk.  `fused=True` skips the assembled
+cache: attention reads the pool and re-encodes K on the fly.  `overlap=True` double-buffers the
 cache and enqueues the gather of chunk i+1 on a second stream; on B200 the persistent
 attention CTAs leave no room for a second resident kernel, so the two do not actually run
 together and the default is off.  Query-side tensors come as one tensor per chunk, [B][layers in chunk][P][T_q][heads][d] (in a model, the queries of a
@@ -21,7 +22,7 @@ from . import binding as ab
 class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
-                 overlap: bool = False, device="cuda"):
+                 overlap: bool = False, fused: bool = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
@@ -36,9 +37,10 @@ class ReusePath:
         self.sel_score = torch.empty((batch, k), dtype=torch.float32, device=device)
         self.ctx_off = torch.empty((batch, k + 1), dtype=torch.int64, device=device)
         self.chunks = [(lb, min(self.nl, lb + self.lpc)) for lb in range(0, self.nl, self.lpc)]
-        self.overlap = bool(overlap) and len(self.chunks) > 1
+        self.fused = bool(fused)
+        self.overlap = bool(overlap) and len(self.chunks) > 1 and not self.fused
         n_ctx = batch * self.lpc * self.ctx_cap * hkv * d
-        n_buf = 2 if self.overlap else 1
+        n_buf = 0 if self.fused else (2 if self.overlap else 1)     # the fused variant has no assembled cache
         self.k_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
         self.v_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
         self.out = [torch.empty((batch, le - lb, self.P, t_q, hq, d), dtype=dt, device=device)
@@ -46,8 +48,8 @@ class ReusePath:
         self.H = torch.empty((batch * self.P,), dtype=torch.float32, device=device)
         self.first_ok = torch.empty((batch,), dtype=torch.int32, device=device)
         self.ws_select = torch.empty(max(256, ab.adapshot_select_workspace_bytes(pool.c.n_shots, batch, k)), **u8)
-        self.ws_attn = torch.empty(max(256, ab.adapshot_attn_workspace_bytes(model, batch, self.P, t_q, self.lpc,
-                                                                              self.ctx_cap)), **u8)
+        ws_fn = ab.adapshot_attn_fused_workspace_bytes if self.fused else ab.adapshot_attn_workspace_bytes
+        self.ws_attn = torch.empty(max(256, ws_fn(model, batch, self.P, t_q, self.lpc, self.ctx_cap)), **u8)
         self.ws_entropy = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(batch * self.P, vocab)), **u8)
         if self.overlap:
             self.side = torch.cuda.Stream(device=device)
@@ -80,6 +82,11 @@ class ReusePath:
                                self.k, self.probes, q, kq, vq, layer_begin, layer_end, out, None,
                                self.ws_attn, self.status)
 
+    def attend_fused(self, q, kq, vq, out, layer_begin: int, layer_end: int):
+        ab.adapshot_query_attn_fused(self.model, self.pool, self.sel_idx, self.ctx_off, self.ctx_cap,
+                                     self.probes, q, kq, vq, layer_begin, layer_end, out, None,
+                                     self.ws_attn, self.status)
+
     def entropy(self, logits: torch.Tensor, tau: float):
         ab.adapshot_entropy(logits, self.H, tau, self.P, self.first_ok, self.ws_entropy, self.status)
 
@@ -88,7 +95,11 @@ class ReusePath:
         gathers of a multi-chunk pass on the side stream, ordered by events).
         q_chunks[i] / kq_chunks[i] / vq_chunks[i] belong to layer chunk self.chunks[i]."""
         self.select(q_emb)
-        if not self.overlap:
+        if self.fused:
+            self.plan()
+            for i, (lb, le) in enumerate(self.chunks):
+                self.attend_fused(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
+        elif not self.overlap:
             for i, (lb, le) in enumerate(self.chunks):
                 self.assemble(lb, le)
                 self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)

@@ -27,13 +27,13 @@ def oracle_path(w, pool, qs, nl, tau):
     return sel, off, np.stack(outs), H, orc.first_ok(H, tau, len(w.probes))
 
 
-def run_gpu_path(w, pool, qs, nl, tau, layers_per_call=None, ctx_cap=None, overlap=False):
+def run_gpu_path(w, pool, qs, nl, tau, layers_per_call=None, ctx_cap=None, overlap=False, fused=False):
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
     dp = hp.dev_pool(ab, pool)
     model = hp.model_of(ab, w, n_layers=nl)
     cap = ctx_cap or w.k * w.len_hi
-    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, cap, layers_per_call, overlap=overlap)
+    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, cap, layers_per_call, overlap=overlap, fused=fused)
     chunk = lambda x: [x[:, lb:le].contiguous().cuda() for lb, le in path.chunks]
     out, H, fo = path.run(qs["q_emb"].cuda(), chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]),
                           qs["logits"].cuda(), tau)
@@ -50,14 +50,14 @@ def _to_bf16_inputs(w, pool, qs):
     return w.scaled(dtype="bf16")
 
 
-def _check(w, nl, layers_per_call=None, tau=None, overlap=False):
+def _check(w, nl, layers_per_call=None, tau=None, overlap=False, fused=False):
     pool, qs = wl.make_pool(w, n_layers=nl), wl.make_queries(w, n_layers=nl)
     if w.dtype == "fp32":     # the attention kernel is bf16: both sides get the same rounded inputs
         w = _to_bf16_inputs(w, pool, qs)
     H_want = orc.entropy(hp.f64(qs["logits"]))
     tau = float(np.median(H_want)) + 1e-2 if tau is None else tau
     sel, off, out_want, H_want, fo_want = oracle_path(w, pool, qs, nl, tau)
-    path, out = run_gpu_path(w, pool, qs, nl, tau, layers_per_call, overlap=overlap)
+    path, out = run_gpu_path(w, pool, qs, nl, tau, layers_per_call, overlap=overlap, fused=fused)
     assert np.array_equal(path.sel_idx.cpu().numpy(), sel)
     assert np.array_equal(path.ctx_off.cpu().numpy(), off)
     err = np.abs(out.cpu().double().numpy() - out_want)
@@ -81,3 +81,19 @@ def test_two_stream_pipeline_three_chunks():
     w = wl.CONFIGS["cfg2"].scaled(n_shots=80, n_layers=3, batch=2, k=20, probes=(5, 20), t_q=32,
                                   vocab=3000, seed=33)
     _check(w, 3, layers_per_call=1, overlap=True)
+
+
+@pytest.mark.parametrize("cfg", ["cfg1", "8b", "d64"])
+def test_fused_variant_whole_path(cfg):
+    # attention straight from the pool, K re-encoded in shared memory: same oracle, same tolerances
+    if cfg == "cfg1":
+        _check(wl.CONFIGS["cfg1"], 1, fused=True)
+    elif cfg == "8b":
+        w = wl.CONFIGS["cfg2"].scaled(n_shots=96, n_layers=3, batch=2, k=24, probes=(3, 6, 12, 24), t_q=48,
+                                      vocab=4000, seed=31)
+        _check(w, 3, layers_per_call=2, fused=True)
+    else:
+        # head_dim 64, T_q > 128 (two own-token tiles), G = 2, 1-token shots among the lengths
+        w = wl.CONFIGS["cfg2"].scaled(n_shots=50, len_lo=1, len_hi=80, n_layers=2, batch=2, k=30, probes=(7, 30),
+                                      t_q=150, head_dim=64, n_q_heads=6, n_kv_heads=3, vocab=2000, seed=35)
+        _check(w, 2, fused=True)
