@@ -102,8 +102,10 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def resolve_workload(name: str, probes_override=None) -> wl.Workload:
+def resolve_workload(name: str, n_layers: int = 0) -> wl.Workload:
     w = wl.CONFIGS[name]
+    if n_layers:          # a stated smaller case of the same shape (profiling captures)
+        w = w.scaled(n_layers=min(w.n_layers, n_layers))
     if w.k == 0:      # cfg4: k = longest similarity-ordered prefix within the token limit; fixed at set-up
         raise SystemExit("cfg4 is a parity configuration; bench workloads: cfg1 cfg2 cfg3 cfg5")
     return w
@@ -263,16 +265,30 @@ def run_ours(args, w: wl.Workload):
     qs = wl.make_queries(wq, dev)
     ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
     lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap)
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc)
+    fused = args.variant == "fused"
+    if fused and not args.layers_per_call:
+        lpc = w.n_layers                      # no assembled cache to fit: all layers in one call
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
     del qs
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    launches_per_step = 2 + (1 if w.n_shots > 8192 else 0) + (1 if path.overlap else 0) + \
-        len(path.chunks) * ((1 if path.overlap else 2) + 3) + 2
+    n_sel = 2 if w.n_shots <= 4096 else (3 if w.n_shots > 8192 else 2)
+    if fused:
+        launches_per_step = n_sel + 1 + len(path.chunks) * 4 + 2
+    else:
+        launches_per_step = n_sel + (1 if path.overlap else 0) + \
+            len(path.chunks) * ((1 if path.overlap else 2) + 3) + 2
+
+    use_graph = args.graph == "on" or (args.graph == "auto" and w.n_layers == 1)
+    if use_graph:
+        path.capture(q_emb, qc, kqc, vqc, logits, args.tau)
 
     def step():
-        path.run(q_emb, qc, kqc, vqc, logits, args.tau)
+        if use_graph:
+            path.replay()
+        else:
+            path.run(q_emb, qc, kqc, vqc, logits, args.tau)
 
     def barrier():
         if dist is not None:
@@ -329,9 +345,16 @@ def run_ours(args, w: wl.Workload):
         marks[1].record()
         mi = 1
         for i, (lb, le) in enumerate(path.chunks):
-            path.assemble(lb, le)
+            if fused:
+                if i == 0:
+                    path.plan()
+            else:
+                path.assemble(lb, le)
             marks[mi + 1].record()
-            path.attend(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
+            if fused:
+                path.attend_fused(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
+            else:
+                path.attend(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
             marks[mi + 2].record()
             mi += 2
         path.entropy(logits, args.tau)
@@ -363,9 +386,10 @@ def run_ours(args, w: wl.Workload):
         "peak_source": f"of {peaks['source']}",
         "traffic": None,
         "ms_per_step": per_call_ms["attn"],
-        "gather": {"bound": "hbm", "achieved": counts["gather_bytes"] / gather_s / 1e9, "peak": peaks["hbm_gbs"],
-                   "unit": "GB/s", "frac": counts["gather_bytes"] / gather_s / 1e9 / peaks["hbm_gbs"],
-                   "ms_per_step": per_call_ms["assemble"], "traffic": None},
+        "gather": None if fused else {
+            "bound": "hbm", "achieved": counts["gather_bytes"] / gather_s / 1e9, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": counts["gather_bytes"] / gather_s / 1e9 / peaks["hbm_gbs"],
+            "ms_per_step": per_call_ms["assemble"], "traffic": None},
         "select": {"bound": "hbm", "achieved": counts["select_bytes"] / (per_call_ms["select"] * 1e-3) / 1e9,
                    "unit": "GB/s", "ms_per_step": per_call_ms["select"]},
         "entropy": {"bound": "hbm", "achieved": counts["entropy_bytes"] / (per_call_ms["entropy"] * 1e-3) / 1e9,
@@ -434,7 +458,7 @@ def run_ours(args, w: wl.Workload):
             "config": {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
                        "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool["n_shots"]),
                        "pool_tokens": int(pool["pool_tokens"]), "ctx_tokens_per_step": counts["ctx_tokens"],
-                       "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
+                       "variant": args.variant, "cuda_graph": use_graph, "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
                        "parallelism": "replicas" if world > 1 else "single"},
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -454,13 +478,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run only the first N layers of the workload (a smaller case for profiler captures)")
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--pool-layers", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
+    ap.add_argument("--variant", default="materialise", choices=["materialise", "fused"],
+                    help="materialise: gather + re-encode into a contiguous cache, then attend; "
+                         "fused: attention reads the pool and re-encodes K in shared memory")
+    ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
+                    help="replay the pass as one CUDA graph (auto: single-layer workloads)")
     ap.add_argument("--tau", type=float, default=0.65)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    w = resolve_workload(args.workload)
+    w = resolve_workload(args.workload, args.layers)
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

@@ -112,7 +112,9 @@ __device__ __forceinline__ uint4 bf16x8_pack(const float* x) {
                     pack_bf16x2(x[6], x[7]));
 }
 
-// One warp per probe token (b, l, j, t): all Hq query heads and Hkv key heads of the
+constexpr int kPrepParts = 4;
+
+// kPrepParts warps per probe token (b, l, j, t): all Hq query heads and Hkv key heads of the
 // token rotate by the same angles (L_j + t) * theta_i.  Block 0 also writes the schedule.
 template <int D>
 __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
@@ -147,7 +149,9 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
     }
   }
   __syncthreads();
-  const long long tok = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long gw = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long tok = gw / kPrepParts;            // kPrepParts warps share the heads of one token
+  const int part = (int)(gw % kPrepParts);
   const long long n_tok = (long long)p.B * p.nl * p.P * p.Tq;
   if (tok >= n_tok) return;
   const int t = (int)(tok % p.Tq);
@@ -169,7 +173,7 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   uint4* kdst = reinterpret_cast<uint4*>(p.kq_rot) + tok * p.Hkv * VPH;
   uint4* qdst_base = reinterpret_cast<uint4*>(p.q_rot);
   const int units = (p.Hq + p.Hkv) * HALF_V;
-  for (int u = lane; u < units; u += 32) {
+  for (int u = part * 32 + lane; u < units; u += 32 * kPrepParts) {
     const int head = u / HALF_V;                    // column == jcol since 32 % HALF_V == 0
     const bool is_q = head < p.Hq;
     const uint4* src = is_q ? qsrc + head * VPH + jcol : ksrc + (head - p.Hq) * VPH + jcol;
@@ -868,6 +872,8 @@ struct CombineParams {
   int B, P, Tq, Hq, Hkv, G, nl, n_mp, n_gangs;
 };
 
+constexpr int kCombineRows = 4;
+
 // Block (q, y): if the range of gang q ends inside a unit that starts in that range, the
 // unit was cut; its pieces sit with gangs q .. q_last.  One warp merges one row.
 template <int D>
@@ -888,40 +894,43 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
   const int q_last = (int)((e_u - 1) / per);
 
   const int lane = threadIdx.x & 31;
-  const int m = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (m >= p.Tq * p.G) return;
-  const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
   const int j = p.P - 1 - pair / p.B, b = pair % p.B;
   const int l = su / p.Hkv, g = su % p.Hkv;
-  const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
   const long long bpj = ((long long)b * p.nl + l) * p.P + j;
-
-  auto slot_row = [&](int qq) -> long long {
-    const int which = (long long)qq * per >= s_u ? 0 : 1;   // the gang's first piece, or its last
-    return (((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x) * kTileM + r;
-  };
-  float M = kNegSentinel;
-  for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[slot_row(qq) * 2]);
   constexpr int EPL = D / 32;                      // output elements per lane
-  float acc[EPL];
+  // kCombineRows rows per warp, unrolled so that the loads of the rows overlap
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  float lsum = 0.f;
-  for (int qq = q; qq <= q_last; ++qq) {
-    const long long sr = slot_row(qq);
-    const float wgt = exp2f(p.ml_part[sr * 2] - M);
-    lsum += p.ml_part[sr * 2 + 1] * wgt;
-    const float* o = p.o_part + sr * D + lane * EPL;
+  for (int rr = 0; rr < kCombineRows; ++rr) {
+    const int m = (blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5)) * kCombineRows + rr;
+    if (m >= p.Tq * p.G) continue;
+    const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
+    const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
+    auto slot_row = [&](int qq) -> long long {
+      const int which = (long long)qq * per >= s_u ? 0 : 1;   // the gang's first piece, or its last
+      return (((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x) * kTileM + r;
+    };
+    float M = kNegSentinel;
+    for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[slot_row(qq) * 2]);
+    float acc[EPL];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] += o[e] * wgt;
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    float lsum = 0.f;
+    for (int qq = q; qq <= q_last; ++qq) {
+      const long long sr = slot_row(qq);
+      const float wgt = exp2f(p.ml_part[sr * 2] - M);
+      lsum += p.ml_part[sr * 2 + 1] * wgt;
+      const float* o = p.o_part + sr * D + lane * EPL;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] += o[e] * wgt;
+    }
+    const float inv = 1.f / lsum;
+    __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D + lane * EPL;
+#pragma unroll
+    for (int e = 0; e < EPL; e += 2)
+      *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+    if (p.lse != nullptr && lane == 0)
+      p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * kLn2;
   }
-  const float inv = 1.f / lsum;
-  __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D + lane * EPL;
-#pragma unroll
-  for (int e = 0; e < EPL; e += 2)
-    *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
-  if (p.lse != nullptr && lane == 0)
-    p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * kLn2;
 }
 
 // ----------------------------------------------------------------- host side
@@ -1082,7 +1091,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   pp.rope_base = model->rope_base;
   for (int i = 0; i < kMaxProbes; ++i) pp.nshots[i] = i < P ? probe_nshots[i] : 0;
   const long long n_tok = (long long)B * nl * P * Tq;
-  attn_prep_kernel<D><<<(unsigned)((n_tok + 7) / 8), 256, 0, st>>>(pp);
+  attn_prep_kernel<D><<<(unsigned)((n_tok * kPrepParts + 7) / 8), 256, 0, st>>>(pp);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   // ---- main kernel
@@ -1127,7 +1136,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   cp.out = ap.out; cp.lse = lse;
   cp.B = B; cp.P = P; cp.Tq = Tq; cp.Hq = Hq; cp.Hkv = Hkv; cp.G = G; cp.nl = nl;
   cp.n_mp = pl.n_mp; cp.n_gangs = n_gangs;
-  const dim3 grid((unsigned)n_gangs, (unsigned)((Tq * G + 7) / 8));
+  const dim3 grid((unsigned)n_gangs, (unsigned)((Tq * G + 8 * kCombineRows - 1) / (8 * kCombineRows)));
   attn_combine_kernel<D><<<grid, 256, 0, st>>>(cp);
   return ads_launch_status();
 }

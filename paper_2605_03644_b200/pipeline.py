@@ -120,3 +120,21 @@ class ReusePath:
                 self.ev_attn[buf].record(main)
         self.entropy(logits, tau)
         return self.out, self.H, self.first_ok
+
+    # ---- the same pass as one CUDA graph: launch-bound small workloads (a few hundred
+    # microseconds per pass) lose a visible share to per-launch host work otherwise
+    def capture(self, q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau: float = 0.65):
+        """Records run(...) on these (static) input tensors into a CUDA graph.  Run one plain
+        pass first (first calls query device attributes).  Returns self; replay() launches it."""
+        if self.overlap:
+            raise ValueError("the two-stream pass is not captured")
+        self.run(q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau)
+        torch.cuda.synchronize()
+        self._graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self._graph):
+            self.run(q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau)
+        return self
+
+    def replay(self):
+        self._graph.replay()
+        return self.out, self.H, self.first_ok

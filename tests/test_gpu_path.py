@@ -97,3 +97,22 @@ def test_fused_variant_whole_path(cfg):
         w = wl.CONFIGS["cfg2"].scaled(n_shots=50, len_lo=1, len_hi=80, n_layers=2, batch=2, k=30, probes=(7, 30),
                                       t_q=150, head_dim=64, n_q_heads=6, n_kv_heads=3, vocab=2000, seed=35)
         _check(w, 2, fused=True)
+
+
+def test_cuda_graph_replay_equals_the_plain_pass():
+    from paper_2605_03644_b200 import binding as ab
+    from paper_2605_03644_b200.pipeline import ReusePath
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=64, batch=1, k=16, probes=(4, 16), t_q=32, vocab=2000, seed=37)
+    pool, qs = wl.make_pool(w), wl.make_queries(w)
+    dp = hp.dev_pool(ab, pool)
+    path = ReusePath(hp.model_of(ab, w), dp, w.batch, w.k, w.probes, w.t_q, w.vocab, w.k * w.len_hi)
+    args = [qs["q_emb"].cuda(), [qs["q"].cuda()], [qs["kq"].cuda()], [qs["vq"].cuda()], qs["logits"].cuda()]
+    path.run(*args)
+    torch.cuda.synchronize()
+    want = (path.out[0].clone(), path.H.clone(), path.sel_idx.clone())
+    path.capture(*args)
+    path.out[0].zero_(); path.H.zero_(); path.sel_idx.zero_()
+    path.replay()
+    torch.cuda.synchronize()
+    assert path.status.item() == 0
+    assert torch.equal(path.out[0], want[0]) and torch.equal(path.H, want[1]) and torch.equal(path.sel_idx, want[2])
