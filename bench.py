@@ -369,14 +369,39 @@ def run_ours(args, w: wl.Workload):
         acc["entropy"] += marks[mi].elapsed_time(marks[mi + 1])
     per_call_ms = {n: acc[n] / n_prof for n in names}
 
-    attn_s = per_call_ms["attn"] * 1e-3
+    # ---- the dominant kernel alone: CUDA events recorded by the library around attn_main_kernel
+    ab.adapshot_profile(True)
+    main_ms = 0.0
+    for _ in range(n_prof):
+        flush.zero_()
+        for i, (lb, le) in enumerate(path.chunks):
+            if fused:
+                if i == 0:
+                    path.plan()
+                path.attend_fused(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
+            else:
+                path.assemble(lb, le)
+                path.attend(qc[i], kqc[i], vqc[i], path.out[i], lb, le)
+            main_ms += ab.adapshot_profile_attn_main_ms()
+    ab.adapshot_profile(False)
+    main_ms /= n_prof
+    n_main = len(path.chunks)
+
+    attn_s = main_ms * 1e-3
     gather_s = per_call_ms["assemble"] * 1e-3
     attn_tflops = counts["attn_flops"] / attn_s / 1e12
     attn_kv_gbs = counts["attn_kv_bytes"] / attn_s / 1e9
     tensor_bound = counts["attn_flops"] / (peaks["bf16_tflops"] * 1e12) >= \
         counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in
+    # profiles/ (cfg3: a 2-layer capture scaled by the layers one launch processes)
+    traffic_attn = {"cfg2": 105.1e6, "cfg3": 2.2425e9 / 2 * path.lpc}.get(w.name) if not fused else None
+    traffic_gather = {"cfg2": 133.8e6, "cfg3": 4.3677e9 / 2 * path.lpc}.get(w.name)
+    if args.layers:
+        traffic_attn = traffic_gather = None
     roofline = {
-        "kernel": "attn_main (per adapshot_query_attn call: prep + main + combine)",
+        "kernel": "attn_main_kernel" + ("<fused>" if fused else ""),
+        "launches_per_step": n_main,
         "bound": "tensor" if tensor_bound else "hbm",
         "achieved": attn_tflops if tensor_bound else attn_kv_gbs,
         "peak": peaks["bf16_tflops"] if tensor_bound else peaks["hbm_gbs"],
@@ -384,12 +409,16 @@ def run_ours(args, w: wl.Workload):
         "frac": (attn_tflops / peaks["bf16_tflops"]) if tensor_bound else (attn_kv_gbs / peaks["hbm_gbs"]),
         "frac_of_sustained_peak": attn_tflops / peaks["bf16_tflops_sustained"] if tensor_bound else None,
         "peak_source": f"of {peaks['source']}",
-        "traffic": None,
-        "ms_per_step": per_call_ms["attn"],
+        "traffic": traffic_attn,
+        "ms_per_launch": main_ms / n_main,
+        "algorithmic_flops_per_launch": counts["attn_flops"] / n_main,
+        "algorithmic_kv_bytes_per_launch": counts["attn_kv_bytes"] / n_main,
+        "whole_call": {"what": "adapshot_query_attn (prep + main + combine)", "ms_per_step": per_call_ms["attn"],
+                       "achieved": counts["attn_flops"] / (per_call_ms["attn"] * 1e-3) / 1e12, "unit": "TFLOP/s"},
         "gather": None if fused else {
             "bound": "hbm", "achieved": counts["gather_bytes"] / gather_s / 1e9, "peak": peaks["hbm_gbs"],
             "unit": "GB/s", "frac": counts["gather_bytes"] / gather_s / 1e9 / peaks["hbm_gbs"],
-            "ms_per_step": per_call_ms["assemble"], "traffic": None},
+            "ms_per_step": per_call_ms["assemble"], "traffic": traffic_gather},
         "select": {"bound": "hbm", "achieved": counts["select_bytes"] / (per_call_ms["select"] * 1e-3) / 1e9,
                    "unit": "GB/s", "ms_per_step": per_call_ms["select"]},
         "entropy": {"bound": "hbm", "achieved": counts["entropy_bytes"] / (per_call_ms["entropy"] * 1e-3) / 1e9,

@@ -208,6 +208,15 @@ ADAPSHOT_API int adapshot_entropy_static(const void* logits, int32_t dtype, int3
                             int64_t row_stride, float* H, float tau, int32_t rows_per_group,
                             int32_t* first_ok, int32_t* status, void* stream);
 
+/* ---- Measurement aid (no counterpart in the paper).  adapshot_profile(1) makes every
+ * later adapshot_query_attn / adapshot_query_attn_fused call record two CUDA events on the
+ * caller's stream around its main (tensor-core) kernel; adapshot_profile_attn_main_ms()
+ * waits for the last such call and returns that kernel's device time in milliseconds
+ * (-1 if none).  Not thread-safe; leave it off (0) outside benchmarks and do not enable
+ * it while a stream is being captured into a graph.                                   */
+ADAPSHOT_API int adapshot_profile(int enable);
+ADAPSHOT_API float adapshot_profile_attn_main_ms(void);
+
 ADAPSHOT_API const char* adapshot_strerror(int code);
 ADAPSHOT_API int adapshot_version(void);
 

@@ -29,6 +29,7 @@ EXPORTS = [
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_static",
+    "adapshot_profile", "adapshot_profile_attn_main_ms",
     "adapshot_strerror", "adapshot_version",
 ]
 
@@ -75,6 +76,18 @@ _attn_fused_ws = _sig("adapshot_attn_fused_workspace_bytes", _sz,
 _attn_fused = _sig("adapshot_query_attn_fused", C.c_int,
                    [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _vp, _i64, _i32, _i32, C.POINTER(_i32), _i32,
                     _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+
+
+_profile = _sig("adapshot_profile", C.c_int, [C.c_int])
+_profile_ms = _sig("adapshot_profile_attn_main_ms", C.c_float, [])
+
+
+def adapshot_profile(enable: bool):
+    _check(_profile(1 if enable else 0))
+
+
+def adapshot_profile_attn_main_ms() -> float:
+    return float(_profile_ms())
 
 
 class AdapshotError(RuntimeError):

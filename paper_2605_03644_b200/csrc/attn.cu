@@ -967,6 +967,11 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
   return r == CUDA_SUCCESS;
 }
 
+// Optional timing of the main kernel alone (adapshot_profile): two events around its launch.
+bool g_profile = false;
+bool g_profile_valid = false;
+cudaEvent_t g_profile_ev[2] = {nullptr, nullptr};
+
 struct AttnPlan {
   int n_mt, n_mp, gang;
   size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, off_rowmap, off_tab, total;
@@ -1104,6 +1109,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   ap.scale_log2 = scale * 1.4426950408889634f;
   const int smem = (int)AttnSmem<128>::kTotal;     // same request for D = 64: one CTA per SM
   static bool attr_done[2][2] = {{false, false}, {false, false}};
+  if (g_profile) ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[0], st));
   if (fused == nullptr) {
     if (!attr_done[0][D == 128]) {
       ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1129,6 +1135,10 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
         tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   }
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  if (g_profile) {
+    ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[1], st));
+    g_profile_valid = true;
+  }
 
   // ---- merge the units that a range boundary cut
   CombineParams cp;
@@ -1230,4 +1240,22 @@ extern "C" int adapshot_query_attn_fused(const adapshot_model_t* model, const ad
                             out, lse, pl, ws, status, st, &src);
   return launch_attn<64>(model, nullptr, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
                          lse, pl, ws, status, st, &src);
+}
+
+extern "C" int adapshot_profile(int enable) {
+  if (enable && g_profile_ev[0] == nullptr) {
+    ADS_CHECK_CUDA(cudaEventCreate(&g_profile_ev[0]));
+    ADS_CHECK_CUDA(cudaEventCreate(&g_profile_ev[1]));
+  }
+  g_profile = enable != 0;
+  g_profile_valid = false;
+  return ADAPSHOT_OK;
+}
+
+extern "C" float adapshot_profile_attn_main_ms(void) {
+  if (!g_profile_valid) return -1.f;
+  float ms = -1.f;
+  if (cudaEventSynchronize(g_profile_ev[1]) != cudaSuccess) return -1.f;
+  if (cudaEventElapsedTime(&ms, g_profile_ev[0], g_profile_ev[1]) != cudaSuccess) return -1.f;
+  return ms;
 }
