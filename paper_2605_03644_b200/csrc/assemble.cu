@@ -8,13 +8,15 @@
 // registers between the 16-byte load and store.  The rotation angles of a token do
 // not depend on layer or head, so each lane forms its few (sin, cos) pairs once per
 // token, in fp64 before the fp32 sincos, and reuses them over heads and layers.
+#include <math.h>
+
 #include "common.cuh"
 
 namespace {
 
 constexpr int kPlanThreads = 256;
 constexpr int kTile = 128;   // the attention kernel reads the cache in 128-token tiles
-constexpr int kRun = 4;      // consecutive destination tokens per warp
+constexpr int kRunMax = 4;   // consecutive destination tokens per warp (fewer when the launch is small)
 
 // One CTA per query: lengths of the selected shots, block-wide exclusive scan.
 __global__ void __launch_bounds__(kPlanThreads)
@@ -105,6 +107,8 @@ struct GatherArgs {
   int k_pos_mode;
   double rope_base;
   int32_t* status;
+  double theta[64];            // theta_i = rope_base^(-2i/D), i < D/2, formed on the host
+  int run;                     // destination tokens per warp and plan lookup
 };
 
 // D = head_dim.  A "pair unit" is the 16-byte vector j of the low half of one head
@@ -127,14 +131,11 @@ gather_rope_kernel(const GatherArgs a) {
   const long long layer_stride_pool = a.pool_tokens * row_vecs;   // in uint4
   const long long layer_stride_ctx = a.ctx_cap * row_vecs;
 
-  // theta_i once per CTA (fp64 pow is slow), then the EPV values of this lane's column
-  __shared__ double theta_sh[D / 2];
-  if (threadIdx.x < D / 2) theta_sh[threadIdx.x] = pow(a.rope_base, -2.0 * (double)threadIdx.x / (double)D);
-  __syncthreads();
+  // the EPV values of theta of this lane's column
   const int jcol = lane % HALF_V;
   double theta[EPV];
 #pragma unroll
-  for (int e = 0; e < EPV; ++e) theta[e] = theta_sh[jcol * EPV + e];
+  for (int e = 0; e < EPV; ++e) theta[e] = a.theta[jcol * EPV + e];
 
   const uint4* kp = static_cast<const uint4*>(a.k_pool);
   const uint4* vp = static_cast<const uint4*>(a.v_pool);
@@ -145,6 +146,7 @@ gather_rope_kernel(const GatherArgs a) {
   // (which selected shot covers the position) is a dependent chain of global loads, so it is
   // done once per run by the whole warp (a 32-ary search: two rounds of parallel probes of the
   // offsets instead of log2(k) serial ones) and then walked forward token by token.
+  const int kRun = a.run;
   const long long runs_per_query = (a.ctx_cap + kRun - 1) / kRun;
   const long long n_runs = (long long)a.B * runs_per_query;
   for (long long run = warp_global; run < n_runs; run += n_warps) {
@@ -264,11 +266,20 @@ gather_rope_kernel(const GatherArgs a) {
 }
 
 template <typename T, int D>
-int launch_gather(const GatherArgs& a, cudaStream_t st) {
-  const long long units = (long long)a.B * ((a.ctx_cap + kRun - 1) / kRun);
+int launch_gather(GatherArgs a, cudaStream_t st) {
   const int warps_per_block = 4;
+  // Resident warps: about six 128-thread CTAs per SM.  Long runs amortise the plan lookup; a
+  // small launch takes shorter runs so that every resident warp gets several and the tail
+  // wave stays short.
+  const long long resident_warps = 148ll * 6 * warps_per_block;
+  const long long tokens = (long long)a.B * a.ctx_cap;
+  a.run = kRunMax;
+  while (a.run > 1 && tokens / a.run < 4 * resident_warps) a.run >>= 1;
+  const long long units = (long long)a.B * ((a.ctx_cap + a.run - 1) / a.run);
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
-  const long long max_blocks = 148ll * 16 * 4;   // a few waves of resident CTAs, grid-stride beyond
+  // measured: one resident wave with a grid-stride loop is best when a run is short (one or two
+  // layers per call), several waves when every run walks many layers
+  const long long max_blocks = a.n_layers_call <= 2 ? 148ll * 6 : 148ll * 16 * 4;
   if (blocks > max_blocks) blocks = max_blocks;
   gather_rope_kernel<T, D><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
   return ads_launch_status();
@@ -322,6 +333,8 @@ extern "C" int adapshot_assemble_kv(const adapshot_model_t* model, const adapsho
   a.n_shots = pool->n_shots; a.B = B; a.k = k; a.n_kv_heads = model->n_kv_heads;
   a.layer_begin = layer_begin; a.n_layers_call = layer_end - layer_begin;
   a.k_pos_mode = model->k_pos_mode; a.rope_base = model->rope_base; a.status = status;
+  for (int i = 0; i < model->head_dim / 2; ++i)
+    a.theta[i] = pow(model->rope_base, -2.0 * (double)i / (double)model->head_dim);
 
   const bool f32 = model->dtype == ADAPSHOT_F32;
   if (model->head_dim == 128)

@@ -87,6 +87,7 @@ struct PrepParams {
   long long ctx_cap;
   int B, k, P, Tq, Hq, Hkv, nl, n_gangs;
   double rope_base;
+  double theta[64];           // theta_i = rope_base^(-2i/D), formed on the host
   int nshots[kMaxProbes];
 };
 
@@ -120,8 +121,6 @@ template <int D>
 __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   constexpr int VPH = D / 8, HALF_V = VPH / 2;
   const int lane = threadIdx.x & 31;
-  __shared__ double theta_sh[D / 2];   // theta_i once per CTA: fp64 pow is slow
-  if (threadIdx.x < D / 2) theta_sh[threadIdx.x] = pow(p.rope_base, -2.0 * (double)threadIdx.x / (double)D);
 
   if (blockIdx.x == 0) {
     Sched* sc = p.sched;
@@ -166,7 +165,7 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   float sn[8], cs[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    rope_sincos(pos, theta_sh[jcol * 8 + e], &sn[e], &cs[e]);
+    rope_sincos(pos, p.theta[jcol * 8 + e], &sn[e], &cs[e]);
   }
   const uint4* qsrc = reinterpret_cast<const uint4*>(p.q) + tok * p.Hq * VPH;
   const uint4* ksrc = reinterpret_cast<const uint4*>(p.kq) + tok * p.Hkv * VPH;
@@ -1094,6 +1093,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   pp.sched = sched; pp.ctx_cap = ctx_cap;
   pp.B = B; pp.k = k; pp.P = P; pp.Tq = Tq; pp.Hq = Hq; pp.Hkv = Hkv; pp.nl = nl; pp.n_gangs = n_gangs;
   pp.rope_base = model->rope_base;
+  for (int i = 0; i < D / 2; ++i) pp.theta[i] = pow(model->rope_base, -2.0 * (double)i / (double)D);
   for (int i = 0; i < kMaxProbes; ++i) pp.nshots[i] = i < P ? probe_nshots[i] : 0;
   const long long n_tok = (long long)B * nl * P * Tq;
   attn_prep_kernel<D><<<(unsigned)((n_tok * kPrepParts + 7) / 8), 256, 0, st>>>(pp);

@@ -100,8 +100,9 @@ class ReusePath:
             for i, (lb, le) in enumerate(self.chunks):
                 self.attend_fused(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
         elif not self.overlap:
+            self.plan()
             for i, (lb, le) in enumerate(self.chunks):
-                self.assemble(lb, le)
+                self.assemble(lb, le, keep_plan=True)
                 self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
         else:
             main = torch.cuda.current_stream()
