@@ -261,7 +261,8 @@ def run_ours(args, w: wl.Workload):
     if n_pool_layers < w.n_layers:
         raise SystemExit("layer aliasing is not implemented; the pool must hold every layer")
     dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
-    model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
+    model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base,
+                          k_pos_mode=args.k_pos_mode)
     qs = wl.make_queries(wq, dev)
     ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
     lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap)
@@ -484,7 +485,7 @@ def run_ours(args, w: wl.Workload):
             "config": {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
                        "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool["n_shots"]),
                        "pool_tokens": int(pool["pool_tokens"]), "ctx_tokens_per_step": counts["ctx_tokens"],
-                       "variant": args.variant, "cuda_graph": use_graph, "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
+                       "variant": args.variant, "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph, "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
                        "parallelism": "replicas" if world > 1 else "single"},
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -512,6 +513,9 @@ def main():
     ap.add_argument("--variant", default="materialise", choices=["materialise", "fused"],
                     help="materialise: gather + re-encode into a contiguous cache, then attend; "
                          "fused: attention reads the pool and re-encodes K in shared memory")
+    ap.add_argument("--k-pos-mode", type=int, default=0, choices=[0, 1],
+                    help="0: pool K carries no position (default); 1: pool K rotated at shot-local positions "
+                         "(the paper's store), the re-encode is one angle per shot")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the pass as one CUDA graph (auto: single-layer workloads)")
     ap.add_argument("--tau", type=float, default=0.65)

@@ -184,6 +184,20 @@ ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, 
                      float* H, float tau, int32_t rows_per_group, int32_t* first_ok,
                      void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
+/* ---- Step 4 over a token subset (Eq. 2 as printed: the entropy over the answer tokens
+ * {Yes, No} of the probe prompt).  subset_ids: device int32 [n_subset] token ids.
+ *   flags 0: p_v is taken from the softmax over the whole vocabulary and not renormalised,
+ *            H = -sum_{v in S} p_v ln p_v  (at most n_subset / e; the case-study values the
+ *            paper prints, two of which exceed ln 2, fit this reading of a two-token set);
+ *   flags 1 (ADAPSHOT_ENTROPY_RENORM): q_v = p_v / sum_S p, H = -sum_S q_v ln q_v <= ln n_subset.
+ * An id outside 0..V-1 is reported as ADAPSHOT_EINDEX in `status` and skipped.  Everything
+ * else (threshold rule, layouts, workspace size) as adapshot_entropy.                      */
+#define ADAPSHOT_ENTROPY_RENORM 1u
+ADAPSHOT_API int adapshot_entropy_subset(const void* logits, int32_t dtype, int32_t R, int32_t V,
+                            int64_t row_stride, const int32_t* subset_ids, int32_t n_subset, uint32_t flags,
+                            float* H, float tau, int32_t rows_per_group, int32_t* first_ok,
+                            void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
 /* ---- adapshot_entropy for callers that cannot provide or allocate scratch.
  * (No counterpart in the paper: this is a packaging variant of the call above.)
  * Meant for callers that must not call cudaMalloc, or hand out workspace, at the

@@ -15,9 +15,11 @@ itself: closed forms, the complex-number form of the rotation, brute-force
 loops, scipy routines, the paper's two-shot position example, and the
 relative-position invariance of rotary attention.
 
-Parity status: every function here is pinned.  (The two-token entropy variant
-of Eq. 2 and the attention-based relevance score of Eq. 5 are not implemented
-here; they are outside the hot path.)
+Parity status: every function here is pinned against closed forms and library
+routines.  entropy_subset (the two-token form of Eq. 2, outside the hot path)
+is pinned as arithmetic, but which of its two readings the paper means is not
+decidable from the text: for that choice it is "parity unpinned".  The
+attention-based relevance score of Eq. 5 is not implemented.
 
 Notation (paper, Sec. 3-4): N shots of lengths T_i, k selected shots, Hq/Hkv
 heads, G = Hq/Hkv, d head_dim, T_q query tokens, L_j context length of probe j.
@@ -230,6 +232,27 @@ def entropy(logits: np.ndarray) -> np.ndarray:
     with np.errstate(divide="ignore", invalid="ignore"):
         terms = np.where(p > 0.0, p * np.log(p), 0.0)
     return -terms.sum(axis=-1)
+
+
+def entropy_subset(logits: np.ndarray, subset_ids, renorm: bool = False) -> np.ndarray:
+    """Eq. 2 as printed: the sum runs over a token subset S (the paper's {Yes, No}).
+
+    renorm False: p = softmax over the whole vocabulary, H = -sum_{v in S} p_v ln p_v.
+    renorm True : q = p restricted to S and renormalised, H = -sum q ln q.
+    (The paper does not say which; two of its printed case-study values exceed ln 2,
+    which a renormalised two-token entropy in nats cannot reach.)
+    """
+    x = np.asarray(logits, dtype=F64)
+    ids = np.asarray(subset_ids, dtype=np.int64)
+    m = x.max(axis=-1, keepdims=True)
+    e = np.exp(x - m)
+    p = e / e.sum(axis=-1, keepdims=True)
+    ps = p[..., ids]
+    if renorm:
+        ps = ps / ps.sum(axis=-1, keepdims=True)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(ps > 0.0, ps * np.log(ps), 0.0)
+    return -t.sum(axis=-1)
 
 
 def first_ok(H: np.ndarray, tau: float, P: int) -> np.ndarray:

@@ -28,7 +28,8 @@ EXPORTS = [
     "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
-    "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_static",
+    "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_subset",
+    "adapshot_entropy_static",
     "adapshot_profile", "adapshot_profile_attn_main_ms",
     "adapshot_strerror", "adapshot_version",
 ]
@@ -61,6 +62,8 @@ _assemble = _sig("adapshot_assemble_kv", C.c_int,
 _entropy_ws = _sig("adapshot_entropy_workspace_bytes", _sz, [_i32, _i32])
 _entropy = _sig("adapshot_entropy", C.c_int,
                 [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _sz, _vp, _vp])
+_entropy_subset = _sig("adapshot_entropy_subset", C.c_int,
+                       [_vp, _i32, _i32, _i32, _i64, _vp, _i32, _u32, _vp, _f, _i32, _vp, _vp, _sz, _vp, _vp])
 _entropy_static = _sig("adapshot_entropy_static", C.c_int,
                        [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _vp])
 _strerror = _sig("adapshot_strerror", C.c_char_p, [C.c_int])
@@ -210,6 +213,18 @@ def adapshot_entropy(logits: torch.Tensor, H: torch.Tensor, tau: float, rows_per
         raise ValueError("logit rows must be contiguous")
     _check(_entropy(logits.data_ptr(), dt, R, V, logits.stride(0), _ptr(H), tau, rows_per_group,
                     _ptr(first_ok), _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_entropy_subset(logits: torch.Tensor, subset_ids: torch.Tensor, H: torch.Tensor, tau: float,
+                            rows_per_group: int, first_ok: Optional[torch.Tensor], ws: torch.Tensor,
+                            status: torch.Tensor, renorm: bool = False):
+    R, V = logits.shape
+    dt = F32 if logits.dtype == torch.float32 else BF16
+    if logits.stride(1) != 1 or subset_ids.dtype != torch.int32:
+        raise ValueError("logit rows must be contiguous and subset_ids int32")
+    _check(_entropy_subset(logits.data_ptr(), dt, R, V, logits.stride(0), _ptr(subset_ids), subset_ids.numel(),
+                           1 if renorm else 0, _ptr(H), tau, rows_per_group, _ptr(first_ok), _ptr(ws),
+                           ws.numel() * ws.element_size(), _ptr(status), _stream()))
 
 
 def adapshot_entropy_static(logits: torch.Tensor, H: torch.Tensor, tau: float, rows_per_group: int,

@@ -147,6 +147,67 @@ entropy_finish_kernel(const float* __restrict__ partial, int n_split, int R, int
   }
 }
 
+// Two-token form of Eq. 2 (the paper takes the entropy over the answer tokens {Yes, No}): like
+// entropy_finish_kernel, but the sum runs over the `n_subset` listed token ids only.
+//   renorm == 0: p_v from the softmax over the whole vocabulary, H = -sum_{v in S} p_v ln p_v
+//   renorm == 1: q_v = p_v / sum_{S} p, H = -sum q_v ln q_v
+template <typename T>
+__global__ void __launch_bounds__(256)
+entropy_subset_finish_kernel(const float* __restrict__ partial, int n_split, int R, int rows_per_group,
+                             const T* __restrict__ logits, long long row_stride, int V,
+                             const int32_t* __restrict__ subset_ids, int n_subset, int renorm,
+                             float tau, float* __restrict__ H, int32_t* __restrict__ first_ok,
+                             int32_t* __restrict__ status) {
+  extern __shared__ float sh_h[];
+  const int g = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  for (int j = warp; j < rows_per_group; j += n_warps) {
+    const int r = g * rows_per_group + j;
+    if (r >= R) break;
+    EntState st{-FLT_MAX, 0.f, 0.f};
+    for (int s = lane; s < n_split; s += 32) {
+      const float* p = partial + 3ll * ((long long)r * n_split + s);
+      st = ent_merge(st, EntState{p[0], p[1], p[2]});
+    }
+    st = ent_warp_reduce(st);
+    const float m = __shfl_sync(0xffffffffu, st.m, 0);
+    const float ln_s = logf(__shfl_sync(0xffffffffu, st.s, 0));
+    const T* row = logits + (long long)r * row_stride;
+    float z = 0.f, u = 0.f, h = 0.f;           // sum e^{x-m}, sum e^{x-m}(x-m), -sum p ln p
+    for (int i = lane; i < n_subset; i += 32) {
+      const int id = subset_ids[i];
+      if (id < 0 || id >= V) {
+        ads_set_status(status, ADAPSHOT_EINDEX);
+        continue;
+      }
+      float x;
+      if constexpr (sizeof(T) == 4) x = row[id]; else x = __bfloat162float(row[id]);
+      const float d = x - m;
+      const float e = __expf(d);
+      z += e;
+      u += e > 0.f ? e * d : 0.f;
+      const float lp = d - ln_s;                // ln p_v
+      const float pv = __expf(lp);
+      h -= pv > 0.f ? pv * lp : 0.f;
+    }
+    z = warp_sum(z); u = warp_sum(u); h = warp_sum(h);
+    if (lane == 0) {
+      float out = renorm ? (z > 0.f ? logf(z) - u / z : 0.f) : h;
+      out = fmaxf(out, 0.f);
+      H[r] = out;
+      sh_h[j] = out;
+    }
+  }
+  __syncthreads();
+  if (first_ok != nullptr && threadIdx.x == 0) {
+    int ok = -1;
+    for (int j = 0; j < rows_per_group && g * rows_per_group + j < R; ++j) {
+      if (sh_h[j] <= tau) { ok = j; break; }
+    }
+    first_ok[g] = ok;
+  }
+}
+
 int ent_splits(int R, int V) {
   // enough CTAs for about two waves of 148 SMs, each slice at least 4096 entries
   int want = (2 * 148 + R - 1) / R;
@@ -192,6 +253,51 @@ extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, in
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   entropy_finish_kernel<<<R / rows_per_group, 256, rows_per_group * sizeof(float), st>>>(
       partial, n_split, R, rows_per_group, tau, H, first_ok);
+  return ads_launch_status();
+}
+
+
+extern "C" int adapshot_entropy_subset(const void* logits, int32_t dtype, int32_t R, int32_t V,
+                                       int64_t row_stride, const int32_t* subset_ids, int32_t n_subset,
+                                       uint32_t flags, float* H, float tau, int32_t rows_per_group,
+                                       int32_t* first_ok, void* ws, size_t ws_bytes, int32_t* status,
+                                       void* stream) {
+  if (logits == nullptr || H == nullptr || ws == nullptr || subset_ids == nullptr) return ADAPSHOT_EINVAL;
+  if (R <= 0 || V <= 0 || row_stride < V || n_subset <= 0 || n_subset > V || (flags & ~1u) != 0)
+    return ADAPSHOT_EINVAL;
+  if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
+  if (rows_per_group <= 0) rows_per_group = 1;
+  if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
+  if (!ads_aligned16(logits) || !ads_aligned16(ws) || (row_stride * es) % 16 != 0 ||
+      ((uintptr_t)subset_ids & 3u))
+    return ADAPSHOT_EALIGN;
+  if (ws_bytes < adapshot_entropy_workspace_bytes(R, V)) return ADAPSHOT_ECAPACITY;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_split = ent_splits(R, V);
+  const int vec = 16 / (int)es;
+  int slice = (V + n_split - 1) / n_split;
+  slice = (slice + vec - 1) / vec * vec;
+  dim3 grid(n_split, R);
+  float* partial = static_cast<float*>(ws);
+  const int renorm = (int)(flags & 1u);
+  const size_t sh = rows_per_group * sizeof(float);
+  if (dtype == ADAPSHOT_F32) {
+    const float* lg = static_cast<const float*>(logits);
+    entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, partial);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+    entropy_subset_finish_kernel<float><<<R / rows_per_group, 256, sh, st>>>(
+        partial, n_split, R, rows_per_group, lg, row_stride, V, subset_ids, n_subset, renorm, tau, H, first_ok,
+        status);
+  } else {
+    const __nv_bfloat16* lg = static_cast<const __nv_bfloat16*>(logits);
+    entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, partial);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+    entropy_subset_finish_kernel<__nv_bfloat16><<<R / rows_per_group, 256, sh, st>>>(
+        partial, n_split, R, rows_per_group, lg, row_stride, V, subset_ids, n_subset, renorm, tau, H, first_ok,
+        status);
+  }
   return ads_launch_status();
 }
 

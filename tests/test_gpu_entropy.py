@@ -79,3 +79,42 @@ def test_entropy_closed_forms_and_threshold():
     assert fo.tolist() == [1]
     H, fo, _ = hp.run_entropy(ab, x[:1].cuda(), 1.0, 1)
     assert fo.tolist() == [-1]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("renorm", [False, True])
+def test_subset_entropy_two_tokens_and_more(dtype, renorm):
+    # the two-token ({Yes, No}) form of Eq. 2 and a larger subset, both readings
+    ab = hp.gpu_binding()
+    g = torch.Generator().manual_seed(9)
+    R, V, P = 8, 32000, 4
+    logits = (torch.randn(R, V, generator=g) * 2.0).to(dtype)
+    for ids in ([9891, 2822], [5, 31999, 17, 4000, 123]):
+        logits[:, ids] += 6.0                       # answer tokens carry visible probability mass
+        ids_t = torch.tensor(ids, dtype=torch.int32, device="cuda")
+        H = torch.full((R,), -1.0, device="cuda")
+        fo = torch.full((R // P,), -7, dtype=torch.int32, device="cuda")
+        ws = torch.empty(max(ab.adapshot_entropy_workspace_bytes(R, V), 256), dtype=torch.uint8, device="cuda")
+        st = hp.new_status()
+        want = orc.entropy_subset(hp.f64(logits), ids, renorm=renorm)
+        tau = float(np.sort(want)[R // 2]) + 1e-3
+        ab.adapshot_entropy_subset(logits.cuda(), ids_t, H, tau, P, fo, ws, st, renorm=renorm)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        got = H.cpu().numpy().astype(np.float64)
+        assert (np.abs(got - want) <= REL_TOL * np.maximum(np.abs(want), 1e-3)).all(), (got, want)
+        if np.abs(want - tau).min() > 1e-4:
+            assert np.array_equal(fo.cpu().numpy(), orc.first_ok(want, tau, P))
+
+
+def test_subset_entropy_reports_a_bad_token_id():
+    ab = hp.gpu_binding()
+    logits = torch.zeros(2, 1000, device="cuda")
+    ids_t = torch.tensor([3, 1000], dtype=torch.int32, device="cuda")
+    H = torch.zeros(2, device="cuda")
+    ws = torch.empty(max(ab.adapshot_entropy_workspace_bytes(2, 1000), 256), dtype=torch.uint8, device="cuda")
+    st = hp.new_status()
+    ab.adapshot_entropy_subset(logits, ids_t, H, 0.5, 1, None, ws, st)
+    torch.cuda.synchronize()
+    assert st.item() == ab.EINDEX
+    assert np.allclose(H.cpu().numpy(), math.log(1000) / 1000, rtol=1e-4)      # the valid token alone

@@ -356,6 +356,37 @@ def test_threshold_rule_on_the_papers_case_study():
     assert (H > math.log(2)).sum() == 2
 
 
+def test_subset_entropy_closed_forms_and_bounds():
+    rng = np.random.default_rng(5)
+    V = 50
+    # uniform logits: every p_v = 1/V, so n tokens give n (1/V) ln V; renormalised: ln n
+    x = np.full((2, V), 0.3)
+    ids = [3, 17, 44]
+    assert np.allclose(orc.entropy_subset(x, ids), 3 * math.log(V) / V, rtol=1e-13)
+    assert np.allclose(orc.entropy_subset(x, ids, renorm=True), math.log(3), rtol=1e-13)
+    # the whole vocabulary as the subset is the full entropy, in either reading
+    y = rng.normal(size=(4, V)) * 2.0
+    assert np.allclose(orc.entropy_subset(y, np.arange(V)), orc.entropy(y), rtol=1e-12)
+    assert np.allclose(orc.entropy_subset(y, np.arange(V), renorm=True), orc.entropy(y), rtol=1e-12)
+    # two tokens with known probabilities: logits ln(0.6), ln(0.3), ln(0.1)
+    z = np.log(np.array([[0.6, 0.3, 0.1]]))
+    want = -(0.6 * math.log(0.6) + 0.3 * math.log(0.3))
+    assert np.allclose(orc.entropy_subset(z, [0, 1]), want, rtol=1e-13)
+    q = np.array([0.6, 0.3]) / 0.9
+    assert np.allclose(orc.entropy_subset(z, [0, 1], renorm=True), -(q * np.log(q)).sum(), rtol=1e-13)
+    assert np.allclose(orc.entropy_subset(z, [0, 1], renorm=True),
+                       scipy.stats.entropy([0.6, 0.3]), rtol=1e-13)          # scipy renormalises itself
+    # bounds: -p ln p <= 1/e per token; renormalised <= ln n; shift invariance
+    ids2 = [1, 7]
+    h = orc.entropy_subset(y, ids2)
+    assert (h >= 0).all() and (h <= 2 / math.e + 1e-15).all()
+    assert (orc.entropy_subset(y, ids2, renorm=True) <= math.log(2) + 1e-15).all()
+    assert np.allclose(orc.entropy_subset(y + 11.0, ids2), h, rtol=1e-12)
+    # the paper's printed two-token values: all within 2/e, two above ln 2 (so not renormalised nats)
+    H = np.array([float(r[1]) for r in _rows("paper_case_study_entropies.txt")])
+    assert (H <= 2 / math.e).all() and (H > math.log(2)).sum() == 2
+
+
 # --------------------------------------------- planted mistakes are caught
 PIN_TESTS = [
     test_rope_hand_value_quarter_turn, test_rope_equals_complex_rotation,
@@ -369,6 +400,7 @@ PIN_TESTS = [
     test_gqa_head_mapping, test_cosine_against_scipy_and_python_sort,
     test_topk_ties_self_match_and_prefix_property,
     test_entropy_closed_forms_and_scipy, test_threshold_rule_on_the_papers_case_study,
+    test_subset_entropy_closed_forms_and_bounds,
 ]
 
 
