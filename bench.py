@@ -189,6 +189,23 @@ def oracle_sample_seconds(w: wl.Workload, pool, qs, row_stride: int):
     return full, desc, measured, float(off[:, -1].sum())
 
 
+def job_aggregate(ms: float, tokens: float, dist, device):
+    """Replicas share nothing but the clock: the job's time is the slowest rank's, its tokens
+    the sum over ranks.  dist = torch.distributed (initialised) or None for one process."""
+    if dist is None:
+        return ms, tokens
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([tokens], device=device, dtype=torch.float64)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item())
+
+
+def rank_seed(seed: int, rank: int) -> int:
+    """Every replica draws its own queries (same pool)."""
+    return seed + 100 * rank if rank else seed
+
+
 def cpu_threads() -> int:
     try:
         import threadpoolctl
@@ -255,7 +272,7 @@ def run_ours(args, w: wl.Workload):
     # ---- resident inputs (every rank: same pool, its own queries)
     n_pool_layers = min(w.n_layers, args.pool_layers) if args.pool_layers else w.n_layers
     pool = wl.make_pool(w, dev, n_layers=n_pool_layers)
-    wq = w.scaled(seed=w.seed + 100 * rank) if rank else w
+    wq = w.scaled(seed=rank_seed(w.seed, rank))
     so = torch.from_numpy(pool["shot_off"]).to(dev)
     k_pool, v_pool = pool["k"], pool["v"]
     if n_pool_layers < w.n_layers:
@@ -319,15 +336,7 @@ def run_ours(args, w: wl.Workload):
         barrier()
     step_ms = np.array([a.elapsed_time(b) for a, b in ev])
     total_ms = float(step_ms.sum())
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        tok = torch.tensor([counts["ctx_tokens"]], device=dev, dtype=torch.float64)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-        job_tokens = float(tok.item())
-    else:
-        job_tokens = counts["ctx_tokens"]
+    total_ms, job_tokens = job_aggregate(total_ms, counts["ctx_tokens"], dist, dev)
     ms_per_step = total_ms / args.steps
     value = job_tokens / (ms_per_step * 1e-3)
     if path.status.item() != 0:
@@ -461,10 +470,7 @@ def run_ours(args, w: wl.Workload):
         b.record()
     barrier()
     e2e_ms = float(np.sum([a.elapsed_time(b) for a, b in ev2]))
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms, _ = job_aggregate(e2e_ms, 0.0, dist, dev)
     e2e_value = job_tokens / (e2e_ms / n_e2e * 1e-3)
 
     # ---- CPU oracle beside it (rank 0, N = 1 only)
