@@ -763,7 +763,9 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
           const float2 neg_m2 = make_float2(-m_used, -m_used);
           float2 part[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-          uint32_t pk[kTileN / 2];
+          // the packed pair c2 goes into the register that held score c2 (already consumed:
+          // c2 <= 2 c2), so the row never needs more than its 128 registers
+          uint32_t* pk = reinterpret_cast<uint32_t*>(s);
 #pragma unroll
           for (int c2 = 0; c2 < kTileN / 2; ++c2) {
             const float2 xs = __ffma2_rn(make_float2(s[2 * c2], s[2 * c2 + 1]), scale2, neg_m2);
