@@ -142,7 +142,8 @@ def planned_ctx_cap(ab, dpool, q_emb, w: wl.Workload) -> int:
 
 
 def algorithmic_counts(w: wl.Workload, ctx_off: np.ndarray, n_layers: int):
-    """Algorithmic bytes / flops of one step from the plan (per the design doc's per-unit figures)."""
+    """Algorithmic bytes / flops of one step from the plan: 2 x bpt bytes per context token and layer
+    for the gather, 4 Hq d flops per (query token, key) and layer for attention."""
     L = ctx_off[:, -1].astype(np.float64)                         # longest probe per query
     Lj = np.stack([ctx_off[:, n] for n in w.probes], axis=1).astype(np.float64)
     bpt = w.bytes_per_token_layer

@@ -231,6 +231,15 @@ ADAPSHOT_API int adapshot_entropy_static(const void* logits, int32_t dtype, int3
 ADAPSHOT_API int adapshot_profile(int enable);
 ADAPSHOT_API float adapshot_profile_attn_main_ms(void);
 
+/* ---- Self-test of the failure path (no counterpart in the paper).  Every wait inside the
+ * attention kernel is bounded: when a barrier is not completed within the limit the CTA
+ * reports ADAPSHOT_ETIMEOUT in `status`, lets its copies land, frees its tensor memory and
+ * returns.  This call runs that wait on a barrier nothing completes, with a limit of about
+ * a millisecond: afterwards `status` holds ADAPSHOT_ETIMEOUT and cycles[0], cycles[1]
+ * (device int64) the SM cycles the two waiting warps spent before giving up.  The kernel
+ * ends normally; the context stays usable.                                               */
+ADAPSHOT_API int adapshot_selftest_wait_timeout(int32_t* status, long long* cycles, void* stream);
+
 ADAPSHOT_API const char* adapshot_strerror(int code);
 ADAPSHOT_API int adapshot_version(void);
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_subset",
     "adapshot_entropy_static",
-    "adapshot_profile", "adapshot_profile_attn_main_ms",
+    "adapshot_profile", "adapshot_profile_attn_main_ms", "adapshot_selftest_wait_timeout",
     "adapshot_strerror", "adapshot_version",
 ]
 
@@ -91,6 +91,13 @@ def adapshot_profile(enable: bool):
 
 def adapshot_profile_attn_main_ms() -> float:
     return float(_profile_ms())
+
+
+_selftest = _sig("adapshot_selftest_wait_timeout", C.c_int, [_vp, _vp, _vp])
+
+
+def adapshot_selftest_wait_timeout(status: torch.Tensor, cycles: torch.Tensor):
+    _check(_selftest(_ptr(status), _ptr(cycles), _stream()))
 
 
 class AdapshotError(RuntimeError):

@@ -934,6 +934,29 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
   }
 }
 
+// Self-test of the bounded wait every pipeline barrier uses: warp 0 waits (with a limit of about a
+// millisecond) on a barrier that nothing will ever complete, gives up, raises the CTA's abort flag
+// and reports ADAPSHOT_ETIMEOUT; warp 1 waits on the same barrier with the long limit and must
+// return as soon as it sees the flag.  The kernel ends normally: the context stays usable.
+__global__ void __launch_bounds__(64) wait_timeout_selftest_kernel(int32_t* status, long long* cycles) {
+  __shared__ __align__(8) unsigned long long barmem;
+  __shared__ int abort_flag[2];
+  const uint32_t b = smem_u32(&barmem);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    abort_flag[0] = abort_flag[1] = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const long long t0 = clock64();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait_limit(b, 0, abort_flag, 2000000ll);
+  if (threadIdx.x == 32) ok = mbar_wait(b, 0, abort_flag);
+  if ((threadIdx.x & 31) == 0) cycles[threadIdx.x >> 5] = ok ? -1 : clock64() - t0;
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag[0] != 0) ads_set_status(status, ADAPSHOT_ETIMEOUT);
+}
+
 // ----------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -1260,4 +1283,10 @@ extern "C" float adapshot_profile_attn_main_ms(void) {
   if (cudaEventSynchronize(g_profile_ev[1]) != cudaSuccess) return -1.f;
   if (cudaEventElapsedTime(&ms, g_profile_ev[0], g_profile_ev[1]) != cudaSuccess) return -1.f;
   return ms;
+}
+
+extern "C" int adapshot_selftest_wait_timeout(int32_t* status, long long* cycles, void* stream) {
+  if (status == nullptr || cycles == nullptr) return ADAPSHOT_EINVAL;
+  wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(status, cycles);
+  return ads_launch_status();
 }
