@@ -51,8 +51,11 @@ class ReusePath:
         ws_fn = ab.adapshot_attn_fused_workspace_bytes if self.fused else ab.adapshot_attn_workspace_bytes
         self.ws_attn = torch.empty(max(256, ws_fn(model, batch, self.P, t_q, self.lpc, self.ctx_cap)), **u8)
         self.ws_entropy = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(batch * self.P, vocab)), **u8)
+        # the entropy probe depends on nothing else in the pass: it runs on a second stream
+        # (a parallel branch when the pass is captured into a graph)
+        self.side = torch.cuda.Stream(device=device)
+        self.ev_begin, self.ev_entropy = torch.cuda.Event(), torch.cuda.Event()
         if self.overlap:
-            self.side = torch.cuda.Stream(device=device)
             self.ev_plan = torch.cuda.Event()
             self.ev_asm = [torch.cuda.Event() for _ in range(2)]
             self.ev_attn = [torch.cuda.Event() for _ in range(2)]
@@ -94,6 +97,12 @@ class ReusePath:
         """One pass of the whole path; everything is enqueued on the current stream (the
         gathers of a multi-chunk pass on the side stream, ordered by events).
         q_chunks[i] / kq_chunks[i] / vq_chunks[i] belong to layer chunk self.chunks[i]."""
+        main = torch.cuda.current_stream()
+        self.ev_begin.record(main)
+        self.side.wait_event(self.ev_begin)
+        with torch.cuda.stream(self.side):
+            self.entropy(logits, tau)
+            self.ev_entropy.record(self.side)
         self.select(q_emb)
         if self.fused:
             self.plan()
@@ -105,7 +114,6 @@ class ReusePath:
                 self.assemble(lb, le, keep_plan=True)
                 self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le)
         else:
-            main = torch.cuda.current_stream()
             self.plan()
             self.ev_plan.record(main)
             self.side.wait_event(self.ev_plan)
@@ -119,7 +127,7 @@ class ReusePath:
                 main.wait_event(self.ev_asm[buf])
                 self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le, buf)
                 self.ev_attn[buf].record(main)
-        self.entropy(logits, tau)
+        main.wait_event(self.ev_entropy)
         return self.out, self.H, self.first_ok
 
     # ---- the same pass as one CUDA graph: launch-bound small workloads (a few hundred
@@ -128,7 +136,7 @@ class ReusePath:
         """Records run(...) on these (static) input tensors into a CUDA graph.  Run one plain
         pass first (first calls query device attributes).  Returns self; replay() launches it."""
         if self.overlap:
-            raise ValueError("the two-stream pass is not captured")
+            raise ValueError("the two-stream gather pass is not captured")
         self.run(q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau)
         torch.cuda.synchronize()
         self._graph = torch.cuda.CUDAGraph()
