@@ -164,11 +164,11 @@ topk_sort_kernel(const double* __restrict__ dots, const double* __restrict__ eno
 
 // Top-k by counting, for pools of up to kRankMaxN shots: the rank of shot i in the order
 // (score descending, id ascending) is the number of shots that precede it; every shot with
-// rank < k writes its id to position rank.  No sort and no serial phases: grid (N / 64, B),
-// 64 candidates per CTA, the comparison range split over four groups of 64 threads.
+// rank < k writes its id to position rank.  No sort and no serial phases: grid (N / 16, B),
+// 16 candidates per CTA, the comparison range split over sixteen groups of 16 threads.
 // "key_j precedes key_i" = key_j < key_i, or equal keys and j < i, = key_j < key_i + (j < i).
 constexpr int kRankMaxN = 4096;
-constexpr int kRankThreads = 256, kRankCand = 64, kRankTile = 2048;
+constexpr int kRankThreads = 256, kRankCand = 16, kRankTile = 2048;
 
 __global__ void __launch_bounds__(kRankThreads)
 rank_topk_kernel(const double* __restrict__ dots, const double* __restrict__ enorm,
