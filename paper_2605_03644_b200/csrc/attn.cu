@@ -18,6 +18,10 @@
 //                 a whole unit stores the final bf16 rows; a range that cuts a unit
 //                 stores un-normalised partials;
 //   attn_combine  log-sum-exp merge of the partials of the cut units.
+// The fused variant (adapshot_query_attn_fused) adds attn_fused_plan (row map and rotary
+// table, once per call) and runs attn_main with two loader warps that copy the context
+// K/V tiles from the pool and re-encode K (Eq. 7) in shared memory, instead of TMA loads
+// from an assembled cache.
 #include <cuda.h>
 #include <float.h>
 

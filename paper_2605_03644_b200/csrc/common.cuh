@@ -38,12 +38,6 @@ __device__ __forceinline__ double warp_sum(double v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-
 // Angle p * theta_i formed in fp64 and reduced to [-pi, pi] before the fp32
 // sincos, so that the result keeps fp32 accuracy at positions of 64K and more.
 __device__ __forceinline__ float rope_reduced_angle(double delta, double theta) {
