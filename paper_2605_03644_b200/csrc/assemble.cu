@@ -277,9 +277,9 @@ int launch_gather(GatherArgs a, cudaStream_t st) {
   while (a.run > 1 && tokens / a.run < 4 * resident_warps) a.run >>= 1;
   const long long units = (long long)a.B * ((a.ctx_cap + a.run - 1) / a.run);
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
-  // measured: one resident wave with a grid-stride loop is best when a run is short (one or two
-  // layers per call), several waves when every run walks many layers
-  const long long max_blocks = a.n_layers_call <= 2 ? 148ll * 6 : 148ll * 16 * 4;
+  // measured: one resident wave with a grid-stride loop is best when a run is short (one
+  // layer per call), several waves when every run walks several layers
+  const long long max_blocks = a.n_layers_call == 1 ? 148ll * 6 : 148ll * 16 * 4;
   if (blocks > max_blocks) blocks = max_blocks;
   gather_rope_kernel<T, D><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
   return ads_launch_status();
