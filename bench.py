@@ -271,13 +271,10 @@ def run_ours(args, w: wl.Workload):
     dev = torch.device("cuda", local)
 
     # ---- resident inputs (every rank: same pool, its own queries)
-    n_pool_layers = min(w.n_layers, args.pool_layers) if args.pool_layers else w.n_layers
-    pool = wl.make_pool(w, dev, n_layers=n_pool_layers)
+    pool = wl.make_pool(w, dev)
     wq = w.scaled(seed=rank_seed(w.seed, rank))
     so = torch.from_numpy(pool["shot_off"]).to(dev)
     k_pool, v_pool = pool["k"], pool["v"]
-    if n_pool_layers < w.n_layers:
-        raise SystemExit("layer aliasing is not implemented; the pool must hold every layer")
     dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base,
                           k_pos_mode=args.k_pos_mode)
@@ -479,7 +476,7 @@ def run_ours(args, w: wl.Workload):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         hpool, hqs = host_inputs(w)
         n_rows = len(w.probes) * w.n_q_heads * w.t_q
-        full, desc, meas, ctx1 = oracle_sample_seconds(w, hpool, hqs, max(1, n_rows // 256))
+        full, desc, meas, ctx1 = oracle_sample_seconds(w, hpool, hqs, max(1, n_rows // 3000))   # about 15 s of oracle work
         cpu_baseline = {"value": ctx1 * w.batch / full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                         "sample": desc, "measured_seconds": meas}
 
@@ -515,7 +512,6 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="run only the first N layers of the workload (a smaller case for profiler captures)")
     ap.add_argument("--layers-per-call", type=int, default=0)
-    ap.add_argument("--pool-layers", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
     ap.add_argument("--variant", default="materialise", choices=["materialise", "fused"],
                     help="materialise: gather + re-encode into a contiguous cache, then attend; "
