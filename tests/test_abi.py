@@ -76,3 +76,17 @@ def test_host_side_argument_checks_launch_nothing(ab):
     assert ent(fake, 0, 1, 8, 4, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EINVAL     # stride < V
     assert ent(fake, 1, 2, 8, 9, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EALIGN     # bf16 row 18 B
     assert ent(fake, 0, 1, 8, 8, fake, 0.5, 1, None, fake, 0, None, None) == ab.ECAPACITY
+
+
+def test_header_is_plain_c(tmp_path):
+    # the boundary is a C ABI: the header must compile as C99 without CUDA or C++
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "t.c"
+    src.write_text('#include "adapshot.h"\nint f(void) { return ADAPSHOT_OK + (int)sizeof(adapshot_model_t); }\n')
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), "-c", str(src),
+                        "-o", str(tmp_path / "t.o")], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
