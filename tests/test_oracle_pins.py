@@ -450,6 +450,18 @@ def _mut_entropy_no_max(logits):
     return -(p * np.log(p)).sum(axis=-1)
 
 
+def _mut_subset_always_renorm(logits, subset_ids, renorm=False):
+    return _ORIG["entropy_subset"](logits, subset_ids, renorm=True)
+
+
+def _mut_subset_local_softmax(logits, subset_ids, renorm=False):
+    # softmax over the subset's logits only, never over the vocabulary
+    x = np.asarray(logits, dtype=np.float64)[..., np.asarray(subset_ids)]
+    e = np.exp(x - x.max(axis=-1, keepdims=True))
+    p = e / e.sum(axis=-1, keepdims=True)
+    return -(p * np.log(p)).sum(axis=-1)
+
+
 def _mut_cosine_no_norm(q_emb, emb):
     return np.asarray(q_emb, dtype=np.float64) @ np.asarray(emb, dtype=np.float64).T
 
@@ -492,6 +504,8 @@ _ORIG = {}
     ("plan_offsets", _mut_plan_inclusive),
     ("entropy", _mut_entropy_log2),
     ("entropy", _mut_entropy_no_max),
+    ("entropy_subset", _mut_subset_always_renorm),
+    ("entropy_subset", _mut_subset_local_softmax),
     ("cosine_scores", _mut_cosine_no_norm),
     ("first_ok", _mut_first_ok_strict),
     ("attn_row", _mut_attn_row_factory("scale")),
@@ -501,7 +515,7 @@ _ORIG = {}
     ("attn_row", _mut_attn_row_factory("prefix")),
 ])
 def test_planted_mistakes_are_caught(name, mutant, monkeypatch):
-    for n in ("rope", "plan_offsets", "entropy"):
+    for n in ("rope", "plan_offsets", "entropy", "entropy_subset"):
         _ORIG[n] = getattr(orc, n)
     assert not _caught(), "pins must pass on the unmodified oracle"
     monkeypatch.setattr(orc, name, mutant)
