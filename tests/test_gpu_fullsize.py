@@ -45,7 +45,7 @@ def _context_of(pool, sel_row, layer, g, L, base):
     return k_ctx[:, None, :], v_rows[:, None, :]      # [L, 1 head, d]
 
 
-def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0):
+def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=False):
     from bench import layers_per_call_for
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
@@ -65,12 +65,12 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0):
     assert orc.min_adjacent_gap(q_emb64, emb64, w.k) > 1e-12
     off = orc.plan_offsets(sel, pool["shot_off"])
     ctx_cap = int(-(-int(off[:, -1].max()) // 128) * 128)
-    lpc = layers_per_call_for(w, ctx_cap)
+    lpc = w.n_layers if fused else layers_per_call_for(w, ctx_cap)
 
     # ---- the CUDA path, as the benchmark launches it
     dpool = ab.Pool(torch.from_numpy(pool["shot_off"]).to(dev), pool["k"], pool["v"], pool["emb"])
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc)
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     tau = 0.65
     path.run(qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"], tau)
@@ -102,6 +102,12 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0):
             errs.append(np.abs(out_l[j, t, h].double().cpu().numpy() - want))
     errs = np.stack(errs)
     assert errs.max() <= MAX_ABS and errs.mean() <= MEAN_ABS, (errs.max(), errs.mean())
+
+    if fused:            # no assembled cache exists in this variant
+        del path, pool, qs, dpool
+        gc.collect()
+        torch.cuda.empty_cache()
+        return
 
     # ---- gather: one layer chunk assembled again (the path reuses the buffer chunk after chunk)
     ci = int(rng.integers(len(path.chunks)))
@@ -150,3 +156,11 @@ def test_cfg4_full_size():
 
 def test_cfg5_full_size():
     _fullsize("cfg5", n_combos=6, rows_per_combo=44)
+
+
+def test_cfg2_full_size_fused_variant():
+    _fullsize("cfg2", n_combos=8, rows_per_combo=32, fused=True)
+
+
+def test_cfg3_full_size_fused_variant():
+    _fullsize("cfg3", fused=True)
