@@ -130,6 +130,62 @@ class ReusePath:
         main.wait_event(self.ev_entropy)
         return self.out, self.H, self.first_ok
 
+    # ---- the same pass for a caller whose tensors live in host memory
+    def run_host(self, host_in: dict, dev_in: dict, host_out: dict, tau: float = 0.65):
+        """One pass with pinned host inputs and pinned host results; no arithmetic here.
+
+        host_in / dev_in: {"q_emb", "logits", "q": [...], "kq": [...], "vq": [...]} (one tensor per
+        layer chunk), the same shapes on both sides; host_out: {"out": [...], "H", "first_ok",
+        "sel_idx"}.  The query-side tensors go up on a copy stream while selection and the
+        gather run, each chunk's output goes down on another while the next chunk is computed,
+        and the logits, the entropy and its results use the side stream: PCIe carries both
+        directions at once and the kernels wait only for the bytes they read.  Everything is
+        joined back to the current stream before returning (the results are complete once that
+        stream is synchronised), so the pass can also be captured into a graph."""
+        if self.overlap:
+            raise ValueError("the two-stream gather pass has no host variant")
+        if not hasattr(self, "h2d"):
+            dev = self.status.device
+            self.h2d, self.d2h = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+            self.ev_in = [torch.cuda.Event() for _ in self.chunks]
+            self.ev_out = [torch.cuda.Event() for _ in self.chunks]
+            self.ev_d2h = torch.cuda.Event()
+        main = torch.cuda.current_stream()
+        self.ev_begin.record(main)
+        for s in (self.side, self.h2d, self.d2h):
+            s.wait_event(self.ev_begin)
+        with torch.cuda.stream(self.side):
+            dev_in["logits"].copy_(host_in["logits"], non_blocking=True)
+            self.entropy(dev_in["logits"], tau)
+            host_out["H"].copy_(self.H, non_blocking=True)
+            host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
+            self.ev_entropy.record(self.side)
+        with torch.cuda.stream(self.h2d):
+            for i in range(len(self.chunks)):
+                for name in ("q", "kq", "vq"):
+                    dev_in[name][i].copy_(host_in[name][i], non_blocking=True)
+                self.ev_in[i].record(self.h2d)
+        dev_in["q_emb"].copy_(host_in["q_emb"], non_blocking=True)
+        self.select(dev_in["q_emb"])
+        self.plan()
+        host_out["sel_idx"].copy_(self.sel_idx, non_blocking=True)
+        for i, (lb, le) in enumerate(self.chunks):
+            if not self.fused:
+                self.assemble(lb, le, keep_plan=True)
+            main.wait_event(self.ev_in[i])
+            if self.fused:
+                self.attend_fused(dev_in["q"][i], dev_in["kq"][i], dev_in["vq"][i], self.out[i], lb, le)
+            else:
+                self.attend(dev_in["q"][i], dev_in["kq"][i], dev_in["vq"][i], self.out[i], lb, le)
+            self.ev_out[i].record(main)
+            with torch.cuda.stream(self.d2h):
+                self.d2h.wait_event(self.ev_out[i])
+                host_out["out"][i].copy_(self.out[i], non_blocking=True)
+        self.ev_d2h.record(self.d2h)
+        main.wait_event(self.ev_d2h)
+        main.wait_event(self.ev_entropy)
+        return host_out
+
     # ---- the same pass as one CUDA graph: launch-bound small workloads (a few hundred
     # microseconds per pass) lose a visible share to per-launch host work otherwise
     def capture(self, q_emb, q_chunks, kq_chunks, vq_chunks, logits, tau: float = 0.65):

@@ -116,3 +116,49 @@ def test_cuda_graph_replay_equals_the_plain_pass():
     torch.cuda.synchronize()
     assert path.status.item() == 0
     assert torch.equal(path.out[0], want[0]) and torch.equal(path.H, want[1]) and torch.equal(path.sel_idx, want[2])
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_host_buffer_pass_equals_the_device_pass(fused):
+    """run_host (pinned host tensors in and out, copies on their own streams) returns what
+    run returns on device tensors, as a plain pass and as a captured graph, three chunks."""
+    from paper_2605_03644_b200 import binding as ab
+    from paper_2605_03644_b200.pipeline import ReusePath
+    nl = 3
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=64, batch=2, k=16, probes=(4, 16), t_q=32, vocab=2000, seed=41)
+    pool, qs = wl.make_pool(w, n_layers=nl), wl.make_queries(w, n_layers=nl)
+    dp = hp.dev_pool(ab, pool)
+    path = ReusePath(hp.model_of(ab, w, n_layers=nl), dp, w.batch, w.k, w.probes, w.t_q, w.vocab,
+                     w.k * w.len_hi, 1, fused=fused)
+    chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
+    host_in = {"q_emb": qs["q_emb"].pin_memory(), "logits": qs["logits"].pin_memory(),
+               "q": [x.pin_memory() for x in chunk(qs["q"])], "kq": [x.pin_memory() for x in chunk(qs["kq"])],
+               "vq": [x.pin_memory() for x in chunk(qs["vq"])]}
+    on_dev = lambda v: [x.cuda() for x in v] if isinstance(v, list) else v.cuda()
+    dev_ref = {n: on_dev(v) for n, v in host_in.items()}
+    path.run(dev_ref["q_emb"], dev_ref["q"], dev_ref["kq"], dev_ref["vq"], dev_ref["logits"])
+    torch.cuda.synchronize()
+    want = {"out": [o.cpu() for o in path.out], "H": path.H.cpu(), "first_ok": path.first_ok.cpu(),
+            "sel_idx": path.sel_idx.cpu()}
+    dev_in = {n: ([torch.zeros_like(x) for x in v] if isinstance(v, list) else torch.zeros_like(v))
+              for n, v in dev_ref.items()}
+    host_out = {n: ([torch.zeros_like(x).pin_memory() for x in v] if isinstance(v, list)
+                    else torch.zeros_like(v).pin_memory()) for n, v in want.items()}
+
+    def same():
+        torch.cuda.synchronize()
+        assert path.status.item() == 0
+        for n, v in want.items():
+            pairs = zip(v, host_out[n]) if isinstance(v, list) else [(v, host_out[n])]
+            assert all(torch.equal(a, b) for a, b in pairs), n
+
+    path.run_host(host_in, dev_in, host_out)
+    same()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        path.run_host(host_in, dev_in, host_out)
+    for v in host_out.values():
+        for x in (v if isinstance(v, list) else [v]):
+            x.zero_()
+    graph.replay()
+    same()
