@@ -36,6 +36,7 @@ constexpr int kMaxProbes = 16;
 constexpr int kMaxPairs = 256;       // (probe, query) pairs one call may hold: B * P <= 256
 constexpr int kMaxCtas = 160;        // persistent grid: one CTA per SM, at most this many
 constexpr int kMaxGang = 8;          // CTAs that share one range of K/V tiles
+constexpr int kUnitCost = 3;         // fixed cost of starting a unit, in tiles (measured: about 10 k clocks)
 constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
 constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
@@ -49,10 +50,12 @@ constexpr float kLn2 = 0.6931471805599453f;
 // Schedule shared by the main and the combine kernel (lives in the workspace).
 // Pairs are ordered longest probe first: pair = (P-1-j) * B + b.  Every pair owns
 // nl * Hkv units (layer, kv head) of n_su tiles each: n_ctx context tiles followed by
-// n_own tiles of the probe's own tokens.
+// n_own tiles of the probe's own tokens.  The ranges are equal in cost, not in tiles: every
+// unit that starts in a range adds kUnitCost tiles' worth of time to it (Q load and pipeline
+// fill, read-out of O), which matters when the units are as short as a range.
 struct Sched {
   long long total;                   // tiles of all units
-  long long per;                     // tiles per gang range
+  long long start[kMaxCtas + 1];     // first tile of every gang's range; start[n_gangs] = total
   long long prefix[kMaxPairs + 1];   // first tile of every pair in the global sequence
   long long Lj[kMaxPairs];           // context length of the pair's probe (clamped to ctx_cap)
   int n_ctx[kMaxPairs];
@@ -148,7 +151,30 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
       }
       sc->prefix[n_pairs] = acc;
       sc->total = acc;
-      sc->per = (acc + p.n_gangs - 1) / p.n_gangs;
+    }
+    __syncthreads();
+    // Range q starts where the cost sequence (every unit preceded by kUnitCost virtual tiles)
+    // reaches q / n_gangs of its length: threads q = 0 .. n_gangs, independently.
+    const long long units_per_pair = (long long)p.nl * p.Hkv;
+    long long vtotal = 0;
+    for (int pi = 0; pi < n_pairs; ++pi) vtotal += (long long)(sc->n_su[pi] + kUnitCost) * units_per_pair;
+    const long long vper = (vtotal + p.n_gangs - 1) / p.n_gangs;
+    for (int q = threadIdx.x; q <= p.n_gangs; q += blockDim.x) {
+      const long long v = (long long)q * vper;
+      long long real = sc->prefix[n_pairs];
+      long long vacc = 0;
+      for (int pi = 0; pi < n_pairs; ++pi) {
+        const long long lv = sc->n_su[pi] + kUnitCost;
+        const long long span = lv * units_per_pair;
+        if (v < vacc + span) {
+          const long long rel = v - vacc;
+          const long long su = rel / lv, off = rel % lv;
+          real = sc->prefix[pi] + su * sc->n_su[pi] + (off > kUnitCost ? off - kUnitCost : 0);
+          break;
+        }
+        vacc += span;
+      }
+      sc->start[q] = real;
     }
   }
   __syncthreads();
@@ -403,8 +429,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   Walker wk0;
-  wk0.begin = (long long)gang_id * sc->per;
-  wk0.end = wk0.begin + sc->per < sc->total ? wk0.begin + sc->per : sc->total;
+  wk0.begin = sc->start[gang_id];
+  wk0.end = sc->start[gang_id + 1];
   wk0.x = wk0.begin;
 
   if (warp == 0) {
@@ -885,9 +911,9 @@ template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p) {
   const Sched* sc = p.sched;
   const int q = blockIdx.x;
-  const long long per = sc->per, total = sc->total;
-  const long long cut = (long long)(q + 1) * per;
-  if (per <= 0 || cut >= total) return;
+  const long long total = sc->total;
+  const long long cut = sc->start[q + 1];
+  if (cut >= total) return;
   const int n_pairs = p.P * p.B;
   const int pair = find_pair(sc, n_pairs, cut);
   const int nsu = sc->n_su[pair];
@@ -895,8 +921,9 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
   if (rel % nsu == 0) return;                       // the cut falls between two units
   const int su = (int)(rel / nsu);
   const long long s_u = sc->prefix[pair] + (long long)su * nsu, e_u = s_u + nsu;
-  if (s_u < (long long)q * per) return;             // an earlier gang holds the unit's first piece
-  const int q_last = (int)((e_u - 1) / per);
+  if (s_u < sc->start[q]) return;                   // an earlier gang holds the unit's first piece
+  int q_last = q + 1;                               // last gang whose range begins inside the unit
+  while (q_last + 1 < p.n_gangs && sc->start[q_last + 1] < e_u) ++q_last;
 
   const int lane = threadIdx.x & 31;
   const int j = p.P - 1 - pair / p.B, b = pair % p.B;
@@ -911,7 +938,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
     const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
     const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
     auto slot_row = [&](int qq) -> long long {
-      const int which = (long long)qq * per >= s_u ? 0 : 1;   // the gang's first piece, or its last
+      const int which = sc->start[qq] >= s_u ? 0 : 1;         // the gang's first piece, or its last
       return (((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x) * kTileM + r;
     };
     float M = kNegSentinel;
