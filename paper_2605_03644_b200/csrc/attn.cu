@@ -36,7 +36,7 @@ constexpr int kMaxProbes = 16;
 constexpr int kMaxPairs = 256;       // (probe, query) pairs one call may hold: B * P <= 256
 constexpr int kMaxCtas = 160;        // persistent grid: one CTA per SM, at most this many
 constexpr int kMaxGang = 8;          // CTAs that share one range of K/V tiles
-constexpr int kUnitCost = 3;         // fixed cost of starting a unit, in tiles (measured: about 10 k clocks)
+constexpr int kUnitCost = 4;          // fixed cost of starting a unit, in tiles (measured: about 10 k clocks)
 constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
 constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
