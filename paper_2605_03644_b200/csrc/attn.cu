@@ -64,7 +64,7 @@ struct Sched {
 
 struct AttnParams {
   const Sched* sched;
-  float* o_part;              // [slots][2][128][D] fp32, un-normalised
+  float* o_part;              // [slots][2][D/4][128][4] fp32, un-normalised (rows contiguous per 4 columns)
   float* ml_part;             // [slots][2][128][2]  (running max in log2 units, row sum)
   __nv_bfloat16* out;         // [B][nl][P][Tq][Hq][D]
   float* lse;                 // [B][nl][P][Hq][Tq] or null
@@ -275,15 +275,19 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
 
 // Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
-template <int D>
+// The fused variant's loader warps take the stages of tile i+1 before they hand over tile i,
+// which needs a third V stage; the room goes at the expense of the read-out staging.
+template <int D, bool FUSED>
 struct AttnSmem {
   static constexpr int kKStages = 2;
-  static constexpr int kVStages = 3;
+  static constexpr int kVStages = FUSED ? 3 : 2;
+  static constexpr uint32_t kStageBytes = FUSED ? 0 : 4096;               // per softmax warp: 32 rows x 128 bytes
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
   static constexpr uint32_t kOffQ = 0;                                    // Q of M tile A, then of M tile B
   static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
   static constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
-  static constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
+  static constexpr uint32_t kOffStage = kOffV + kVStages * kTileBytes;    // read-out staging of the 8 softmax warps
+  static constexpr uint32_t kOffBar = kOffStage + 8 * kStageBytes;
   static constexpr uint32_t kTotal = kOffBar + 512 + 1024;               // barriers + alignment slack
 };
 
@@ -377,13 +381,14 @@ __global__ void __launch_bounds__(FUSED ? kFusedThreads : kAttnThreads, 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
                  const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
-  using SM = AttnSmem<D>;
+  using SM = AttnSmem<D, FUSED>;
   constexpr int SUB = D / 64;
   constexpr int KS = SM::kKStages, VS = SM::kVStages;
   constexpr uint32_t kTileBytes = SM::kTileBytes;
   constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, 0);
   constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, 1);
   constexpr uint32_t kTmemS = 0, kTmemO = 256;
+  constexpr int kSoftmaxWarp0 = FUSED ? 4 : 2;          // first of the eight softmax warps
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -735,7 +740,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     cp_async_wait<0>();
   } else {
     // ---------------------------------------------------- softmax + read-out of O
-    const int x = (warp - (FUSED ? 4 : 2)) >> 2;   // 0: M tile A, 1: M tile B
+    const int x = (warp - kSoftmaxWarp0) >> 2;     // 0: M tile A, 1: M tile B
     const int quarter = warp & 3;                  // TMEM lanes this warp may touch
     const int r = quarter * 32 + lane;             // row of the M tile
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
@@ -825,61 +830,106 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const bool row_ok = m < p.Tq * p.G;
         if (w.n_tiles == 0) {
           // nothing of this M pair falls into the piece: a neutral partial (a whole unit is never empty)
-          if (row_ok) {
-            float* orow = p.o_part + ((w.slot * 2 + x) * kTileM + r) * D;
+          float4* otile = reinterpret_cast<float4*>(p.o_part) + (w.slot * 2 + x) * (long long)(D / 4) * kTileM + r;
 #pragma unroll
-            for (int e = 0; e < D; e += 4) *reinterpret_cast<float4*>(orow + e) = make_float4(0.f, 0.f, 0.f, 0.f);
-            float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
-            ml[0] = kNegSentinel;
-            ml[1] = 0.f;
-          }
+          for (int c4 = 0; c4 < D / 4; ++c4) otile[c4 * kTileM] = make_float4(0.f, 0.f, 0.f, 0.f);
+          float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
+          ml[0] = kNegSentinel;
+          ml[1] = 0.f;
           continue;
         }
         ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull + x), ni & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         if (w.whole) {
-          // the piece covers the unit: normalise and store the final rows
+          // The piece covers the unit: normalise and store the final rows.  A thread owns a
+          // row, and rows are far apart in the output, so a direct store would touch 32 lines
+          // per instruction; instead the warp passes 64 columns at a time through its staging
+          // area (16-byte chunks swizzled by the row) and writes four rows' 128-byte segments
+          // per instruction.
           const float inv = 1.f / l_sum;
-          const int t = t_row, hh = m % p.G, h = w.g * p.G + hh;
           const long long bpj = w.outer_own;
-          __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D;
+          unsigned char* stg = base_ptr + SM::kOffStage + (warp - kSoftmaxWarp0) * SM::kStageBytes;
+          const int sub = lane >> 3, ch = lane & 7;            // read-back: row 4 j + sub, chunk ch
+          const int m0 = mt * kTileM + quarter * 32;
+          if constexpr (FUSED) {
+            // (no staging area in the fused variant's shared-memory plan: one row per thread)
+            const int hq = w.g * p.G + m % p.G;
+            __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t_row) * p.Hq) + hq) * (long long)D;
 #pragma unroll
-          for (int q4 = 0; q4 < D / 32; ++q4) {
-            float o[32];
-            tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
-            if (row_ok) {
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+              float o[32];
+              tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
+              if (q4 == D / 32 - 1) {
+                tc_fence_before();
+                mbar_arrive(bar(kBarOEmpty + x));
+              }
+              if (row_ok) {
 #pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                float v8[8];
+                for (int e = 0; e < 32; e += 8) {
+                  float v8[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v8[u] = o[e + u] * inv;
-                *reinterpret_cast<uint4*>(dst + q4 * 32 + e) = bf16x8_pack(v8);
+                  for (int u = 0; u < 8; ++u) v8[u] = o[e + u] * inv;
+                  *reinterpret_cast<uint4*>(dst + q4 * 32 + e) = bf16x8_pack(v8);
+                }
               }
             }
+          } else {
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h) {
+            float o[64];
+            tmem_ld32(o_addr + h * 64, reinterpret_cast<uint32_t*>(o));
+            tmem_ld32(o_addr + h * 64 + 32, reinterpret_cast<uint32_t*>(o + 32));
+            if (h == D / 64 - 1) {             // O is in registers: the next item may overwrite it
+              tc_fence_before();
+              mbar_arrive(bar(kBarOEmpty + x));
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              float v8[8];
+#pragma unroll
+              for (int u = 0; u < 8; ++u) v8[u] = o[c * 8 + u] * inv;
+              *reinterpret_cast<uint4*>(stg + lane * 128 + ((c ^ (lane & 7)) << 4)) = bf16x8_pack(v8);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int row = 4 * j + sub;
+              const int mm = m0 + row;
+              const uint4 v = *reinterpret_cast<const uint4*>(stg + row * 128 + ((ch ^ (row & 7)) << 4));
+              if (mm < p.Tq * p.G) {
+                const int tt = mm / p.G, hq = w.g * p.G + mm % p.G;
+                __nv_bfloat16* dst = p.out + (((bpj * p.Tq + tt) * p.Hq) + hq) * (long long)D;
+                *reinterpret_cast<uint4*>(dst + h * 64 + ch * 8) = v;
+              }
+            }
+            __syncwarp();
           }
-          if (row_ok && p.lse != nullptr)
-            p.lse[(bpj * p.Hq + h) * p.Tq + t] = (m_used + log2f(l_sum)) * kLn2;
+          }
+          if (row_ok && p.lse != nullptr) {
+            const int hh = m % p.G, hq = w.g * p.G + hh;
+            p.lse[(bpj * p.Hq + hq) * p.Tq + t_row] = (m_used + log2f(l_sum)) * kLn2;
+          }
         } else {
-          float* orow = p.o_part + ((w.slot * 2 + x) * kTileM + r) * D;
+          // un-normalised partial, four columns of 128 rows at a time ([D/4][128][4] per M tile):
+          // a warp's 32 rows are 512 contiguous bytes per store
+          float4* otile = reinterpret_cast<float4*>(p.o_part) + (w.slot * 2 + x) * (long long)(D / 4) * kTileM + r;
 #pragma unroll
           for (int q4 = 0; q4 < D / 32; ++q4) {
             float o[32];
             tmem_ld32(o_addr + q4 * 32, reinterpret_cast<uint32_t*>(o));
-            if (row_ok) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<float4*>(orow + q4 * 32 + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+            if (q4 == D / 32 - 1) {
+              tc_fence_before();
+              mbar_arrive(bar(kBarOEmpty + x));
             }
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              otile[(q4 * 8 + e / 4) * kTileM] = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
           }
-          if (row_ok) {
-            float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
-            ml[0] = m_used;
-            ml[1] = l_sum;
-          }
+          float* ml = p.ml_part + ((w.slot * 2 + x) * kTileM + r) * 2;
+          ml[0] = m_used;
+          ml[1] = l_sum;
         }
-        tc_fence_before();
-        mbar_arrive(bar(kBarOEmpty + x));
         ++ni;
       }
     }
@@ -903,10 +953,10 @@ struct CombineParams {
   int B, P, Tq, Hq, Hkv, G, nl, n_mp, n_gangs;
 };
 
-constexpr int kCombineRows = 4;
+constexpr int kCombineRows = 8;      // rows per warp
 
 // Block (q, y): if the range of gang q ends inside a unit that starts in that range, the
-// unit was cut; its pieces sit with gangs q .. q_last.  One warp merges one row.
+// unit was cut; its pieces sit with gangs q .. q_last.  One warp merges eight rows.
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p) {
   const Sched* sc = p.sched;
@@ -929,40 +979,50 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
   const int j = p.P - 1 - pair / p.B, b = pair % p.B;
   const int l = su / p.Hkv, g = su % p.Hkv;
   const long long bpj = ((long long)b * p.nl + l) * p.P + j;
-  constexpr int EPL = D / 32;                      // output elements per lane
-  // kCombineRows rows per warp, unrolled so that the loads of the rows overlap
+  // A warp merges 8 rows: lane = (row r_sub, 4-column chunk c_sub of the 16 columns of one
+  // step), so that a load is 8 rows x 16 bytes contiguous per chunk in the partial layout
+  // ([D/4][128 rows][4] per M tile) and a store fills one 32-byte sector per row.
+  const int r_sub = lane & 7, c_sub = lane >> 3;
+  const int m = (blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5)) * kCombineRows + r_sub;
+  if (m >= p.Tq * p.G) return;
+  const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
+  const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
+  auto slot_tile = [&](int qq) -> long long {
+    const int which = sc->start[qq] >= s_u ? 0 : 1;           // the gang's first piece, or its last
+    return ((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x;
+  };
+  float M = kNegSentinel;
+  for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[(slot_tile(qq) * kTileM + r) * 2]);
+  const float4* o4 = reinterpret_cast<const float4*>(p.o_part);
+  float4 acc[D / 16];
 #pragma unroll
-  for (int rr = 0; rr < kCombineRows; ++rr) {
-    const int m = (blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5)) * kCombineRows + rr;
-    if (m >= p.Tq * p.G) continue;
-    const int mt = m / kTileM, r = m % kTileM, mp = mt >> 1, x = mt & 1;
-    const int t = m / p.G, hh = m % p.G, h = g * p.G + hh;
-    auto slot_row = [&](int qq) -> long long {
-      const int which = sc->start[qq] >= s_u ? 0 : 1;         // the gang's first piece, or its last
-      return (((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x) * kTileM + r;
-    };
-    float M = kNegSentinel;
-    for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[slot_row(qq) * 2]);
-    float acc[EPL];
+  for (int it = 0; it < D / 16; ++it) acc[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+  float lsum = 0.f;
+  for (int qq = q; qq <= q_last; ++qq) {
+    const long long tile = slot_tile(qq);
+    const float* ml = p.ml_part + (tile * kTileM + r) * 2;
+    const float wgt = exp2f(ml[0] - M);
+    lsum += ml[1] * wgt;
+    float4 v[D / 16];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    float lsum = 0.f;
-    for (int qq = q; qq <= q_last; ++qq) {
-      const long long sr = slot_row(qq);
-      const float wgt = exp2f(p.ml_part[sr * 2] - M);
-      lsum += p.ml_part[sr * 2 + 1] * wgt;
-      const float* o = p.o_part + sr * D + lane * EPL;
+    for (int it = 0; it < D / 16; ++it) v[it] = o4[(tile * (D / 4) + it * 4 + c_sub) * kTileM + r];
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[e] += o[e] * wgt;
+    for (int it = 0; it < D / 16; ++it) {
+      acc[it].x += v[it].x * wgt; acc[it].y += v[it].y * wgt;
+      acc[it].z += v[it].z * wgt; acc[it].w += v[it].w * wgt;
     }
-    const float inv = 1.f / lsum;
-    __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D + lane * EPL;
-#pragma unroll
-    for (int e = 0; e < EPL; e += 2)
-      *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
-    if (p.lse != nullptr && lane == 0)
-      p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * kLn2;
   }
+  const float inv = 1.f / lsum;
+  __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t) * p.Hq) + h) * (long long)D;
+#pragma unroll
+  for (int it = 0; it < D / 16; ++it) {
+    uint2 packed;
+    packed.x = pack_bf16x2(acc[it].x * inv, acc[it].y * inv);
+    packed.y = pack_bf16x2(acc[it].z * inv, acc[it].w * inv);
+    *reinterpret_cast<uint2*>(dst + (it * 4 + c_sub) * 4) = packed;
+  }
+  if (p.lse != nullptr && c_sub == 0)
+    p.lse[(bpj * p.Hq + h) * p.Tq + t] = (M + log2f(lsum)) * kLn2;
 }
 
 // Self-test of the bounded wait every pipeline barrier uses: warp 0 waits (with a limit of about a
@@ -1163,7 +1223,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   ap.n_mt = pl.n_mt; ap.n_mp = pl.n_mp; ap.gang = pl.gang; ap.n_gangs = n_gangs;
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
-  const int smem = (int)AttnSmem<128>::kTotal;     // same request for D = 64: one CTA per SM
+  const int smem = (int)AttnSmem<128, false>::kTotal;     // same request for D = 64 and for the fused variant: one CTA per SM
   static bool attr_done[2][2] = {{false, false}, {false, false}};
   if (g_profile) ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[0], st));
   if (fused == nullptr) {
