@@ -56,6 +56,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct Sched {
   long long total;                   // tiles of all units
   long long start[kMaxCtas + 1];     // first tile of every gang's range; start[n_gangs] = total
+  int first_pair[kMaxCtas + 1];      // pair that holds start[q]
   long long prefix[kMaxPairs + 1];   // first tile of every pair in the global sequence
   long long Lj[kMaxPairs];           // context length of the pair's probe (clamped to ctx_cap)
   int n_ctx[kMaxPairs];
@@ -158,11 +159,11 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
     const long long units_per_pair = (long long)p.nl * p.Hkv;
     long long vtotal = 0;
     for (int pi = 0; pi < n_pairs; ++pi) vtotal += (long long)(sc->n_su[pi] + kUnitCost) * units_per_pair;
-    const long long vper = (vtotal + p.n_gangs - 1) / p.n_gangs;
     for (int q = threadIdx.x; q <= p.n_gangs; q += blockDim.x) {
-      const long long v = (long long)q * vper;
+      const long long v = (long long)q * vtotal / p.n_gangs;
       long long real = sc->prefix[n_pairs];
       long long vacc = 0;
+      int fp = n_pairs - 1;
       for (int pi = 0; pi < n_pairs; ++pi) {
         const long long lv = sc->n_su[pi] + kUnitCost;
         const long long span = lv * units_per_pair;
@@ -170,11 +171,13 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
           const long long rel = v - vacc;
           const long long su = rel / lv, off = rel % lv;
           real = sc->prefix[pi] + su * sc->n_su[pi] + (off > kUnitCost ? off - kUnitCost : 0);
+          fp = pi;
           break;
         }
         vacc += span;
       }
       sc->start[q] = real;
+      sc->first_pair[q] = fp;
     }
   }
   __syncthreads();
@@ -288,7 +291,7 @@ struct AttnSmem {
   static constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
   static constexpr uint32_t kOffStage = kOffV + kVStages * kTileBytes;    // read-out staging of the 8 softmax warps
   static constexpr uint32_t kOffBar = kOffStage + 8 * kStageBytes;
-  static constexpr uint32_t kTotal = kOffBar + 512 + 1024;               // barriers + alignment slack
+  static constexpr uint32_t kTotal = kOffBar + 256 + 1024 + 1024;        // barriers, schedule cache, alignment slack
 };
 
 // mbarrier slots (8 bytes each)
@@ -307,7 +310,38 @@ struct Piece {
 
 struct Walker {
   long long x, begin, end;
+  int pair;                      // pair that holds x (pieces only move forward)
 };
+
+// The part of the schedule a CTA walks, copied to shared memory once: the pairs from the
+// one its range starts in.  Pairs beyond the copy (a range that spans more than
+// kCachePairs pairs) are read from the workspace.
+constexpr int kCachePairs = 40;
+struct SchedCache {
+  long long prefix[kCachePairs + 1];
+  long long Lj[kCachePairs];
+  int n_ctx[kCachePairs];
+  int n_su[kCachePairs];
+  long long begin, end;
+  int p0, n;
+};
+static_assert(sizeof(SchedCache) <= 1024, "the schedule cache has 1 KiB of shared memory");
+struct PairInfo {
+  long long prefix, next_prefix, Lj;
+  int n_ctx, n_su;
+};
+__device__ __forceinline__ PairInfo pair_info(const Sched* sc, const SchedCache* c, int pair) {
+  PairInfo pi;
+  const int k = pair - c->p0;
+  if (k >= 0 && k < c->n) {
+    pi.prefix = c->prefix[k]; pi.next_prefix = c->prefix[k + 1]; pi.Lj = c->Lj[k];
+    pi.n_ctx = c->n_ctx[k]; pi.n_su = c->n_su[k];
+  } else {
+    pi.prefix = sc->prefix[pair]; pi.next_prefix = sc->prefix[pair + 1]; pi.Lj = sc->Lj[pair];
+    pi.n_ctx = sc->n_ctx[pair]; pi.n_su = sc->n_su[pair];
+  }
+  return pi;
+}
 
 __device__ __forceinline__ int find_pair(const Sched* sc, int n_pairs, long long x) {
   int lo = 0, hi = n_pairs;
@@ -318,19 +352,22 @@ __device__ __forceinline__ int find_pair(const Sched* sc, int n_pairs, long long
   return lo;
 }
 
-__device__ __forceinline__ bool next_piece(const Sched* sc, int n_pairs, Walker& wk, Piece& pc) {
+__device__ __forceinline__ bool next_piece(const Sched* sc, const SchedCache* cache, int n_pairs, Walker& wk,
+                                           Piece& pc) {
   if (wk.x >= wk.end) return false;
-  const int lo = find_pair(sc, n_pairs, wk.x);
-  const int nsu = sc->n_su[lo];
-  const long long rel = wk.x - sc->prefix[lo];
+  PairInfo pi = pair_info(sc, cache, wk.pair);
+  while (wk.pair + 1 < n_pairs && pi.next_prefix <= wk.x) pi = pair_info(sc, cache, ++wk.pair);
+  const int lo = wk.pair;
+  const int nsu = pi.n_su;
+  const long long rel = wk.x - pi.prefix;
   pc.pair = lo;
   pc.su = (int)(rel / nsu);
   pc.t0 = (int)(rel % nsu);
   const long long room = wk.end - wk.x;
   pc.t1 = (int)(room < (long long)(nsu - pc.t0) ? pc.t0 + room : nsu);
   pc.n_su = nsu;
-  pc.n_ctx = sc->n_ctx[lo];
-  pc.Lj = sc->Lj[lo];
+  pc.n_ctx = pi.n_ctx;
+  pc.Lj = pi.Lj;
   pc.first_of_gang = wk.x == wk.begin;
   wk.x += pc.t1 - pc.t0;
   return true;
@@ -428,15 +465,36 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
     tmem_relinquish();
   }
+  // the CTA's part of the schedule, fetched by two otherwise idle warps while the rest is set up
+  SchedCache* cache = reinterpret_cast<SchedCache*>(base_ptr + SM::kOffBar + 256);
+  if (warp >= 2 && warp < 4) {
+    const int p0 = sc->first_pair[gang_id];
+    const int n = min(kCachePairs, n_pairs - p0);
+    for (int k = threadIdx.x - 64; k <= n; k += 64) {
+      cache->prefix[k] = sc->prefix[p0 + k];
+      if (k < n) {
+        cache->Lj[k] = sc->Lj[p0 + k];
+        cache->n_ctx[k] = sc->n_ctx[p0 + k];
+        cache->n_su[k] = sc->n_su[p0 + k];
+      }
+    }
+    if (threadIdx.x == 64) {
+      cache->begin = sc->start[gang_id];
+      cache->end = sc->start[gang_id + 1];
+      cache->p0 = p0;
+      cache->n = n;
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   Walker wk0;
-  wk0.begin = sc->start[gang_id];
-  wk0.end = sc->start[gang_id + 1];
+  wk0.begin = cache->begin;
+  wk0.end = cache->end;
   wk0.x = wk0.begin;
+  wk0.pair = cache->p0;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -446,7 +504,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       bool ok = true;
       Walker wk = wk0;
       Piece pc;
-      while (ok && next_piece(sc, n_pairs, wk, pc)) {
+      while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
         for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
           Item w;
           make_item(p, pc, gang_id, mp, w);
@@ -555,7 +613,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         return true;
       };
-      while (ok && next_piece(sc, n_pairs, wk, pc)) {
+      while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
         for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
           Item w;
           make_item(p, pc, gang_id, mp, w);
@@ -705,7 +763,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
     };
-    while (ok && next_piece(sc, n_pairs, wk, pc)) {
+    while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
       for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
         Item w;
         make_item(p, pc, gang_id, mp, w);
@@ -750,7 +808,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     bool ok = true;
     Walker wk = wk0;
     Piece pc;
-    while (ok && next_piece(sc, n_pairs, wk, pc)) {
+    while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
       for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
         Item w;
         make_item(p, pc, gang_id, mp, w);
@@ -991,14 +1049,18 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const CombineParams p
     const int which = sc->start[qq] >= s_u ? 0 : 1;           // the gang's first piece, or its last
     return ((long long)(2 * qq + which) * p.n_mp + mp) * 2 + x;
   };
+  // (when there are fewer tiles than gangs, empty ranges lie between the pieces)
+  auto has_piece = [&](int qq) -> bool { return sc->start[qq] < sc->start[qq + 1]; };
   float M = kNegSentinel;
-  for (int qq = q; qq <= q_last; ++qq) M = fmaxf(M, p.ml_part[(slot_tile(qq) * kTileM + r) * 2]);
+  for (int qq = q; qq <= q_last; ++qq)
+    if (has_piece(qq)) M = fmaxf(M, p.ml_part[(slot_tile(qq) * kTileM + r) * 2]);
   const float4* o4 = reinterpret_cast<const float4*>(p.o_part);
   float4 acc[D / 16];
 #pragma unroll
   for (int it = 0; it < D / 16; ++it) acc[it] = make_float4(0.f, 0.f, 0.f, 0.f);
   float lsum = 0.f;
   for (int qq = q; qq <= q_last; ++qq) {
+    if (!has_piece(qq)) continue;
     const long long tile = slot_tile(qq);
     const float* ml = p.ml_part + (tile * kTileM + r) * 2;
     const float wgt = exp2f(ml[0] - M);
