@@ -400,7 +400,7 @@ def run_ours(args, w: wl.Workload):
         counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in
     # profiles/ (cfg3: a 2-layer capture scaled by the layers one launch processes)
-    traffic_attn = {"cfg2": 103.9e6, "cfg3": 2.2422e9 / 2 * path.lpc}.get(w.name) if not fused else None
+    traffic_attn = {"cfg2": 104.3e6, "cfg3": 2.2407e9 / 2 * path.lpc}.get(w.name) if not fused else None
     traffic_gather = {"cfg2": 123.5e6, "cfg3": 4.2670e9 / 2 * path.lpc}.get(w.name)
     if args.layers:
         traffic_attn = traffic_gather = None
