@@ -124,16 +124,21 @@ __device__ __forceinline__ uint4 bf16x8_pack(const float* x) {
 constexpr int kPrepParts = 4;
 
 // kPrepParts warps per probe token (b, l, j, t): all Hq query heads and Hkv key heads of the
-// token rotate by the same angles (L_j + t) * theta_i.  Block 0 also writes the schedule.
+// token rotate by the same angles (L_j + t) * theta_i.  The last block writes the schedule instead.
 template <int D>
 __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   constexpr int VPH = D / 8, HALF_V = VPH / 2;
   const int lane = threadIdx.x & 31;
 
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == gridDim.x - 1) {
+    // the schedule, by a block of its own (beside the rotation, not in front of a share of it);
+    // intermediate values stay in shared memory
+    __shared__ long long s_pre[kMaxPairs + 1], s_vpre[kMaxPairs + 1];
+    __shared__ int s_nsu[kMaxPairs];
     Sched* sc = p.sched;
     const int n_pairs = p.P * p.B;
     const int n_own = (p.Tq + kTileN - 1) / kTileN;
+    const long long units_per_pair = (long long)p.nl * p.Hkv;
     for (int pi = threadIdx.x; pi < n_pairs; pi += blockDim.x) {
       const int j = p.P - 1 - pi / p.B, b = pi % p.B;
       long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
@@ -142,45 +147,48 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
       sc->Lj[pi] = Lj;
       sc->n_ctx[pi] = n_ctx;
       sc->n_su[pi] = n_ctx + n_own;
+      s_nsu[pi] = n_ctx + n_own;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-      long long acc = 0;
+      long long acc = 0, vacc = 0;
       for (int pi = 0; pi < n_pairs; ++pi) {
+        s_pre[pi] = acc;
+        s_vpre[pi] = vacc;
         sc->prefix[pi] = acc;
-        acc += (long long)sc->n_su[pi] * p.nl * p.Hkv;
+        acc += (long long)s_nsu[pi] * units_per_pair;
+        vacc += (long long)(s_nsu[pi] + kUnitCost) * units_per_pair;
       }
+      s_pre[n_pairs] = acc;
+      s_vpre[n_pairs] = vacc;
       sc->prefix[n_pairs] = acc;
       sc->total = acc;
     }
     __syncthreads();
     // Range q starts where the cost sequence (every unit preceded by kUnitCost virtual tiles)
     // reaches q / n_gangs of its length: threads q = 0 .. n_gangs, independently.
-    const long long units_per_pair = (long long)p.nl * p.Hkv;
-    long long vtotal = 0;
-    for (int pi = 0; pi < n_pairs; ++pi) vtotal += (long long)(sc->n_su[pi] + kUnitCost) * units_per_pair;
+    const long long vtotal = s_vpre[n_pairs];
     for (int q = threadIdx.x; q <= p.n_gangs; q += blockDim.x) {
       const long long v = (long long)q * vtotal / p.n_gangs;
-      long long real = sc->prefix[n_pairs];
-      long long vacc = 0;
+      long long real = s_pre[n_pairs];
       int fp = n_pairs - 1;
-      for (int pi = 0; pi < n_pairs; ++pi) {
-        const long long lv = sc->n_su[pi] + kUnitCost;
-        const long long span = lv * units_per_pair;
-        if (v < vacc + span) {
-          const long long rel = v - vacc;
-          const long long su = rel / lv, off = rel % lv;
-          real = sc->prefix[pi] + su * sc->n_su[pi] + (off > kUnitCost ? off - kUnitCost : 0);
-          fp = pi;
-          break;
+      if (v < vtotal) {
+        int lo = 0, hi = n_pairs;                   // pair with s_vpre[lo] <= v < s_vpre[lo + 1]
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (s_vpre[mid] <= v) lo = mid; else hi = mid;
         }
-        vacc += span;
+        const long long lv = s_nsu[lo] + kUnitCost;
+        const long long rel = v - s_vpre[lo];
+        const long long su = rel / lv, off = rel % lv;
+        real = s_pre[lo] + su * s_nsu[lo] + (off > kUnitCost ? off - kUnitCost : 0);
+        fp = lo;
       }
       sc->start[q] = real;
       sc->first_pair[q] = fp;
     }
+    return;
   }
-  __syncthreads();
   const long long gw = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long tok = gw / kPrepParts;            // kPrepParts warps share the heads of one token
   const int part = (int)(gw % kPrepParts);
@@ -1274,7 +1282,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   for (int i = 0; i < D / 2; ++i) pp.theta[i] = pow(model->rope_base, -2.0 * (double)i / (double)D);
   for (int i = 0; i < kMaxProbes; ++i) pp.nshots[i] = i < P ? probe_nshots[i] : 0;
   const long long n_tok = (long long)B * nl * P * Tq;
-  attn_prep_kernel<D><<<(unsigned)((n_tok * kPrepParts + 7) / 8), 256, 0, st>>>(pp);
+  attn_prep_kernel<D><<<(unsigned)((n_tok * kPrepParts + 7) / 8) + 1, 256, 0, st>>>(pp);   // + the schedule block
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   // ---- main kernel
