@@ -13,10 +13,27 @@ namespace {
 constexpr int kSortCap = 8192;      // candidates one CTA sorts in shared memory
 constexpr int kSortThreads = 1024;
 
-// One warp per pool row i: dots[b][i] = <q_b, e_i> for all b, enorm[i] = |e_i|.
+// Order-preserving map of an fp64 score to an unsigned key; larger score -> SMALLER
+// key so that an ascending sort on (key, id) lists the most relevant shot first and
+// equal scores by ascending id.
+__device__ __forceinline__ unsigned long long desc_key(double s) {
+  unsigned long long u = (unsigned long long)__double_as_longlong(s);
+  u = (u >> 63) ? ~u : (u | 0x8000000000000000ull);   // ascending in s
+  return ~u;
+}
+__device__ __forceinline__ double key_score(unsigned long long k) {
+  unsigned long long u = ~k;
+  u = (u >> 63) ? (u & 0x7fffffffffffffffull) : ~u;
+  return __longlong_as_double((long long)u);
+}
+
+// One warp per pool row i: dots[b][i] = <q_b, e_i> for all b, enorm[i] = |e_i|.  With
+// keys_out set (pools that the rank kernel handles) the warp also forms |q_b| from the values
+// it loads anyway and writes the sort key of cos(q_b, e_i) in place of the dot product, so
+// that the ranking kernel's CTAs do not each redo N fp64 divisions.
 __global__ void __launch_bounds__(256)
 cosine_dots_kernel(const float* __restrict__ emb, const float* __restrict__ q_emb, int N, int E,
-                   int B, double* __restrict__ dots, double* __restrict__ enorm) {
+                   int B, double* __restrict__ dots, double* __restrict__ enorm, int keys_out) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= N) return;
@@ -35,33 +52,31 @@ cosine_dots_kernel(const float* __restrict__ emb, const float* __restrict__ q_em
   if (lane == 0) enorm[row] = sqrt(nn);
   for (int b = 0; b < B; ++b) {
     const float* q = q_emb + (long long)b * E;
-    double acc = 0.0;
+    double acc = 0.0, qq = 0.0;
     if (vec_ok) {
       for (int i = lane * 4; i < E; i += 128) {
         float4 v = *reinterpret_cast<const float4*>(e + i);   // L1-resident after the first pass
         float4 w = __ldg(reinterpret_cast<const float4*>(q + i));
         acc += (double)v.x * w.x + (double)v.y * w.y + (double)v.z * w.z + (double)v.w * w.w;
+        qq += (double)w.x * w.x + (double)w.y * w.y + (double)w.z * w.z + (double)w.w * w.w;
       }
     } else {
-      for (int i = lane; i < E; i += 32) acc += (double)e[i] * q[i];
+      for (int i = lane; i < E; i += 32) {
+        acc += (double)e[i] * q[i];
+        qq += (double)q[i] * q[i];
+      }
     }
     acc = warp_sum(acc);
-    if (lane == 0) dots[(long long)b * N + row] = acc;
+    if (keys_out) {
+      qq = warp_sum(qq);
+      if (lane == 0) {
+        const double den = sqrt(qq) * sqrt(nn);
+        reinterpret_cast<unsigned long long*>(dots)[(long long)b * N + row] = desc_key(den > 0.0 ? acc / den : 0.0);
+      }
+    } else if (lane == 0) {
+      dots[(long long)b * N + row] = acc;
+    }
   }
-}
-
-// Order-preserving map of an fp64 score to an unsigned key; larger score -> SMALLER
-// key so that an ascending sort on (key, id) lists the most relevant shot first and
-// equal scores by ascending id.
-__device__ __forceinline__ unsigned long long desc_key(double s) {
-  unsigned long long u = (unsigned long long)__double_as_longlong(s);
-  u = (u >> 63) ? ~u : (u | 0x8000000000000000ull);   // ascending in s
-  return ~u;
-}
-__device__ __forceinline__ double key_score(unsigned long long k) {
-  unsigned long long u = ~k;
-  u = (u >> 63) ? (u & 0x7fffffffffffffffull) : ~u;
-  return __longlong_as_double((long long)u);
 }
 
 __device__ __forceinline__ bool pair_less(unsigned long long ka, int ia, unsigned long long kb, int ib) {
@@ -171,35 +186,14 @@ constexpr int kRankMaxN = 4096;
 constexpr int kRankThreads = 256, kRankCand = 16, kRankTile = 2048;
 
 __global__ void __launch_bounds__(kRankThreads)
-rank_topk_kernel(const double* __restrict__ dots, const double* __restrict__ enorm,
-                 const float* __restrict__ q_emb, int E, int N, int k,
+rank_topk_kernel(const unsigned long long* __restrict__ all_keys, int N, int k,
                  int32_t* __restrict__ final_idx, float* __restrict__ final_score) {
   __shared__ unsigned long long keys[kRankTile];
-  __shared__ double red[kRankThreads / 32];
-  __shared__ double qnorm_sh;
   __shared__ int part_cnt[kRankThreads];
   const int b = blockIdx.y;
   const int tid = threadIdx.x;
-  {
-    const float* q = q_emb + (long long)b * E;
-    double acc = 0.0;
-    for (int i = tid; i < E; i += kRankThreads) acc += (double)q[i] * q[i];
-    acc = warp_sum(acc);
-    if ((tid & 31) == 0) red[tid >> 5] = acc;
-    __syncthreads();
-    if (tid < 32) {
-      double v = tid < kRankThreads / 32 ? red[tid] : 0.0;
-      v = warp_sum(v);
-      if (tid == 0) qnorm_sh = sqrt(v);
-    }
-    __syncthreads();
-  }
-  const double qn = qnorm_sh;
-  auto key_of = [&](int j) -> unsigned long long {
-    const double den = qn * enorm[j];
-    const double sc = den > 0.0 ? dots[(long long)b * N + j] / den : 0.0;
-    return desc_key(sc);
-  };
+  const unsigned long long* gkeys = all_keys + (long long)b * N;
+  auto key_of = [&](int j) -> unsigned long long { return gkeys[j]; };
   const int i = blockIdx.x * kRankCand + (tid & (kRankCand - 1));
   const int part = tid / kRankCand;                       // which quarter of every tile this thread scans
   const unsigned long long ki = i < N ? key_of(i) : ~0ull;
@@ -277,12 +271,13 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
 
   const int warps_per_block = 8;
   cosine_dots_kernel<<<(N + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
-      pool->emb, q_emb, N, E, B, dots, enorm);
+      pool->emb, q_emb, N, E, B, dots, enorm, N <= kRankMaxN ? 1 : 0);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   if (N <= kRankMaxN) {
     dim3 grid((N + kRankCand - 1) / kRankCand, B);
-    rank_topk_kernel<<<grid, kRankThreads, 0, st>>>(dots, enorm, q_emb, E, N, k, sel_idx, sel_score);
+    rank_topk_kernel<<<grid, kRankThreads, 0, st>>>(reinterpret_cast<const unsigned long long*>(dots), N, k, sel_idx,
+                                                    sel_score);
     return ads_launch_status();
   }
 
