@@ -6,17 +6,18 @@
 //   attn_prep     rotates Q and the probe's own K to their positions L_j + t, packs the
 //                 Q rows of one KV head (GQA) into an M-major tile layout, and writes
 //                 the schedule (how many 128-key tiles every (probe, query) pair has
-//                 and how the tile sequence is cut into equal ranges);
+//                 and where the tile sequence is cut into ranges of equal cost);
 //   attn_main     persistent CTAs.  A CTA works on two 128-row M tiles of one KV head
 //                 at a time ("M pair"): TMA stages each K/V tile once for both, one
 //                 thread issues tcgen05 UMMAs (S = Q K^T, O += P V, accumulators in
 //                 TMEM, P kept in TMEM), two groups of four warps run the online
 //                 softmax of the two M tiles (one thread per row) and alternate on the
-//                 tensor pipe.  The global tile sequence is cut into equal ranges, one
-//                 per gang of CTAs (the CTAs of a gang take the M pairs of the same
-//                 K/V tiles, so the tiles are shared through L2).  A range that covers
-//                 a whole unit stores the final bf16 rows; a range that cuts a unit
-//                 stores un-normalised partials;
+//                 tensor pipe.  The global tile sequence is cut into ranges of equal
+//                 cost, one per gang of CTAs (the CTAs of a gang take the M pairs of the
+//                 same K/V tiles, so the tiles are shared through L2).  A range that
+//                 covers a whole unit stores the final bf16 rows (staged through shared
+//                 memory into whole row segments); a range that cuts a unit stores
+//                 un-normalised partials;
 //   attn_combine  log-sum-exp merge of the partials of the cut units.
 // The fused variant (adapshot_query_attn_fused) adds attn_fused_plan (row map and rotary
 // table, once per call) and runs attn_main with two loader warps that copy the context
