@@ -255,6 +255,31 @@ def entropy_subset(logits: np.ndarray, subset_ids, renorm: bool = False) -> np.n
     return -t.sum(axis=-1)
 
 
+def probe_rounds(H_by_round, schedule, tau: float):
+    """Multi-round probing (Sec. 4.1; the case study of Sec. 5 runs it with rounds 4..16 and
+    20..32 and tau = 0.65): rounds are probed in order, and a query's answer is the first
+    shot count, in schedule order, whose entropy is at most tau.
+    H_by_round[r] is [B][m] (entropies of round r's m probes), schedule[r] the m shot
+    counts.  Returns per query (round, probe index, shot count), (-1, -1, -1) when no probe
+    meets the threshold, and the number of rounds that had to be run for the whole batch."""
+    B = np.asarray(H_by_round[0], dtype=F64).shape[0]
+    stops = [(-1, -1, -1)] * B
+    rounds_run = 0
+    for r, Hr in enumerate(H_by_round):
+        rounds_run = r + 1
+        Hr = np.asarray(Hr, dtype=F64)
+        for b in range(B):
+            if stops[b][0] >= 0:
+                continue
+            for j in range(Hr.shape[1]):
+                if Hr[b, j] <= tau:
+                    stops[b] = (r, j, int(schedule[r][j]))
+                    break
+        if all(s[0] >= 0 for s in stops):
+            break
+    return stops, rounds_run
+
+
 def first_ok(H: np.ndarray, tau: float, P: int) -> np.ndarray:
     """Per group of P nested probes: index of the first probe with H <= tau,
     -1 if none (the minimum shot count that satisfies the threshold)."""

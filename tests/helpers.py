@@ -84,3 +84,9 @@ def bf16_ulp_diff(a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
 
 
 f64 = wl.to_f64
+
+
+def golden(name: str) -> str:
+    """Path of a fixture under tests/golden."""
+    import os
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)

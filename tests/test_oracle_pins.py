@@ -356,6 +356,26 @@ def test_threshold_rule_on_the_papers_case_study():
     assert (H > math.log(2)).sum() == 2
 
 
+def test_probe_rounds_on_the_papers_case_study():
+    rows = _rows("paper_case_study_entropies.txt")
+    shots = [int(r[0]) for r in rows]
+    H = np.array([float(r[1]) for r in rows])
+    schedule = [shots[:4], shots[4:]]
+    stops, rounds_run = orc.probe_rounds([H[None, :4], H[None, 4:]], schedule, 0.65)
+    assert stops == [(1, 2, 28)] and rounds_run == 2          # the paper: second round, 28 shots
+    # a second query that is satisfied by the very first probe does not shorten the batch's
+    # rounds, and a query that is never satisfied reports -1
+    H2 = np.stack([H, np.concatenate([[0.1], H[1:]]), np.full(8, 0.9)])
+    stops, rounds_run = orc.probe_rounds([H2[:, :4], H2[:, 4:]], schedule, 0.65)
+    assert stops == [(1, 2, 28), (0, 0, 4), (-1, -1, -1)] and rounds_run == 2
+    # with only the satisfied query, one round is enough
+    stops, rounds_run = orc.probe_rounds([H2[1:2, :4], H2[1:2, 4:]], schedule, 0.65)
+    assert stops == [(0, 0, 4)] and rounds_run == 1
+    # the threshold is inclusive
+    stops, _ = orc.probe_rounds([np.array([[0.65, 0.2]])], [[3, 6]], 0.65)
+    assert stops == [(0, 0, 3)]
+
+
 def test_subset_entropy_closed_forms_and_bounds():
     rng = np.random.default_rng(5)
     V = 50
@@ -400,7 +420,7 @@ PIN_TESTS = [
     test_gqa_head_mapping, test_cosine_against_scipy_and_python_sort,
     test_topk_ties_self_match_and_prefix_property,
     test_entropy_closed_forms_and_scipy, test_threshold_rule_on_the_papers_case_study,
-    test_subset_entropy_closed_forms_and_bounds,
+    test_subset_entropy_closed_forms_and_bounds, test_probe_rounds_on_the_papers_case_study,
 ]
 
 
@@ -472,6 +492,24 @@ def _mut_first_ok_strict(H, tau, P):
                      for b in range(Hm.shape[0])], dtype=np.int32)
 
 
+def _mut_probe_rounds_lowest_entropy(H_by_round, schedule, tau):
+    # takes the probe with the lowest entropy under the threshold, not the first one
+    stops, rounds_run = _ORIG["probe_rounds"](H_by_round, schedule, tau)
+    out = []
+    for b, (r, j, n) in enumerate(stops):
+        if r >= 0:
+            Hr = np.asarray(H_by_round[r])[b]
+            j = int(np.argmin(Hr))
+            n = int(schedule[r][j])
+        out.append((r, j, n))
+    return out, rounds_run
+
+
+def _mut_probe_rounds_runs_every_round(H_by_round, schedule, tau):
+    stops, _ = _ORIG["probe_rounds"](H_by_round, schedule, tau)
+    return stops, len(H_by_round)
+
+
 def _mut_attn_row_factory(kind):
     def f(q_row, kq, vq, k_ctx, v_ctx, L_j, t, kv_head, base, scale=None):
         d = q_row.shape[-1]
@@ -508,6 +546,8 @@ _ORIG = {}
     ("entropy_subset", _mut_subset_local_softmax),
     ("cosine_scores", _mut_cosine_no_norm),
     ("first_ok", _mut_first_ok_strict),
+    ("probe_rounds", _mut_probe_rounds_lowest_entropy),
+    ("probe_rounds", _mut_probe_rounds_runs_every_round),
     ("attn_row", _mut_attn_row_factory("scale")),
     ("attn_row", _mut_attn_row_factory("qpos")),
     ("attn_row", _mut_attn_row_factory("causal")),
@@ -515,7 +555,7 @@ _ORIG = {}
     ("attn_row", _mut_attn_row_factory("prefix")),
 ])
 def test_planted_mistakes_are_caught(name, mutant, monkeypatch):
-    for n in ("rope", "plan_offsets", "entropy", "entropy_subset"):
+    for n in ("rope", "plan_offsets", "entropy", "entropy_subset", "probe_rounds"):
         _ORIG[n] = getattr(orc, n)
     assert not _caught(), "pins must pass on the unmodified oracle"
     monkeypatch.setattr(orc, name, mutant)
