@@ -72,9 +72,9 @@ class Workload:
         return replace(self, **kw)
 
 
-# The five configurations named by the build's baseline file.  Items the
-# baseline leaves open: emb_dim of cfg4/cfg5 (1024), vocab of cfg4/cfg5
-# (128256), sigma of the lognormal of cfg5 (0.4).
+# The five benchmark configurations.  Values their description leaves open and that are
+# fixed here: emb_dim of cfg4/cfg5 (1024), vocab of cfg4/cfg5 (128256), sigma of the
+# lognormal of cfg5's shot lengths (0.4).
 CONFIGS = {
     "cfg1": Workload("cfg1", 1, 4, 1, 64, 1e4, "fp32", 64, "const", 32, 32, 128,
                      1, 8, (8,), 16, 1024, "fp32", seed=0, channel_scale=False,
