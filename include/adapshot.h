@@ -161,8 +161,10 @@ ADAPSHOT_API int adapshot_query_attn(const adapshot_model_t* model,
  * by one fp32 complex multiplication; K' rounded once to bf16 as in the materialised
  * path).  ctx_off: the plan written by adapshot_assemble_kv (plan-only call is enough)
  * for the same sel_idx; ctx_cap: an upper bound of every L (sizes the workspace: a row
- * map of B * ctx_cap int32 and a table of ctx_cap * d * 4 bytes).  Needs
- * model->k_pos_mode == 0, pool_tokens < 2^31.  Other arguments as above.             */
+ * maps of 2 * B * ctx_cap int32 and a table of ctx_cap * d * 4 bytes).  Both
+ * k_pos_mode values are taken (1: every key of a shot is rotated by the angle of the
+ * shot's first position, read from the same table).  Needs pool_tokens < 2^31.  Other
+ * arguments as above.                                                                */
 ADAPSHOT_API size_t adapshot_attn_fused_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
                                            int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap);
 ADAPSHOT_API int adapshot_query_attn_fused(const adapshot_model_t* model, const adapshot_pool_t* pool,

@@ -80,6 +80,8 @@ struct AttnParams {
   const __nv_bfloat16* kq_rot;   // [B*nl*P][Tq][Hkv][D], rotated by the prep kernel
   const __nv_bfloat16* vq;
   const int* row_map;            // [B][ctx_cap]: pool token of every context position, -1 beyond L
+  const int* off_map;            // [B][ctx_cap]: first position of the shot a position lies in (k_pos_mode 1)
+  int k_pos_mode;                // 0: angle = position; 1: angle = the shot's first position (Eq. 7 as printed)
   const float2* rope_tab;        // [ctx_cap rounded up to 128][D/2]: (cos, sin) of position * theta_i
   long long pool_tokens, ctx_cap;
   int layer_begin;
@@ -247,6 +249,7 @@ struct FusedPlanParams {
   const int32_t* sel_idx;     // [B][k]
   const long long* shot_off;  // [n_shots+1]
   int* row_map;               // [B][ctx_cap]
+  int* off_map;               // [B][ctx_cap]: first position of the position's shot
   float2* rope_tab;           // [tab_rows][D/2]
   long long ctx_cap, tab_rows;
   int B, k, n_shots, half_d;
@@ -262,7 +265,7 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
       const int b = (int)(u / p.ctx_cap);
       const long long pos = u % p.ctx_cap;
       const long long* off = p.ctx_off + (long long)b * (p.k + 1);
-      int row = -1;
+      int row = -1, first = 0;
       if (pos < off[p.k]) {
         int lo = 0, hi = p.k;          // shot slot with off[lo] <= pos < off[lo+1]
         while (hi - lo > 1) {
@@ -271,8 +274,10 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
         }
         const int s = p.sel_idx[(long long)b * p.k + lo];
         if (s >= 0 && s < p.n_shots) row = (int)(p.shot_off[s] + (pos - off[lo]));
+        first = (int)off[lo];
       }
       p.row_map[u] = row;
+      p.off_map[u] = first;
     } else {
       const long long v = u - n_map;
       const long long pos = v / p.half_d;
@@ -740,18 +745,26 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       unsigned char* kt = base_ptr + SM::kOffK + sk * kTileBytes;
       const long long pos0 = (long long)(w.ctx_begin + i) * kTileN + row0;
       float2 cur[8];
-      const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + pos0 * (D / 2) + jj * 8);
+      auto load_angles = [&](long long table_row) {
+        const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + table_row * (D / 2) + jj * 8);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float4 t4 = tab[e];
-        cur[2 * e] = make_float2(t4.x, t4.y);
-        cur[2 * e + 1] = make_float2(t4.z, t4.w);
-      }
+        for (int e = 0; e < 4; ++e) {
+          const float4 t4 = tab[e];
+          cur[2 * e] = make_float2(t4.x, t4.y);
+          cur[2 * e + 1] = make_float2(t4.z, t4.w);
+        }
+      };
+      const bool per_shot = p.k_pos_mode == 1;     // the angle is that of the shot's first position
+      if (!per_shot) load_angles(pos0);
 #pragma unroll
       for (int u = 0; u < PAIRS; ++u) {
         const int row = row0 + u * kRowStep;
         uint4* lo = reinterpret_cast<uint4*>(kt + chunk_addr(row, 0));
         uint4* hi = reinterpret_cast<uint4*>(kt + chunk_addr(row, 1));
+        if (per_shot) {
+          const long long pos = pos0 + u * kRowStep;
+          load_angles(pos < p.ctx_cap ? p.off_map[(long long)w.b * p.ctx_cap + pos] : 0);
+        }
         float x[8], y[8], xr[8], yr[8];
         bf16x8_unpack(*lo, x);
         bf16x8_unpack(*hi, y);
@@ -762,7 +775,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         *lo = bf16x8_pack(xr);
         *hi = bf16x8_pack(yr);
-        if (u + 1 < PAIRS) {
+        if (!per_shot && u + 1 < PAIRS) {
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const float c = cur[e].x * step[e].x - cur[e].y * step[e].y;
@@ -1160,7 +1173,7 @@ cudaEvent_t g_profile_ev[2] = {nullptr, nullptr};
 
 struct AttnPlan {
   int n_mt, n_mp, gang;
-  size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, off_rowmap, off_tab, total;
+  size_t off_qrot, off_kqrot, off_sched, off_opart, off_ml, off_rowmap, off_offmap, off_tab, total;
   long long tab_rows;
 };
 
@@ -1188,11 +1201,12 @@ AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, 
   pl.off_sched = off; off += ads_round_up(sizeof(Sched), 256);
   pl.off_opart = off; off += ads_round_up(slots * 2 * kTileM * D * 4, 256);
   pl.off_ml = off;    off += ads_round_up(slots * 2 * kTileM * 2 * 4, 256);
-  pl.off_rowmap = pl.off_tab = off;
+  pl.off_rowmap = pl.off_offmap = pl.off_tab = off;
   pl.tab_rows = 0;
   if (fused_ctx_cap > 0) {
     pl.tab_rows = (fused_ctx_cap + kTileN - 1) / kTileN * kTileN;
     pl.off_rowmap = off; off += ads_round_up((size_t)B * fused_ctx_cap * 4, 256);
+    pl.off_offmap = off; off += ads_round_up((size_t)B * fused_ctx_cap * 4, 256);
     pl.off_tab = off;    off += ads_round_up((size_t)pl.tab_rows * (D / 2) * 8, 256);
   }
   pl.total = off;
@@ -1256,13 +1270,14 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
 
   // ---- fused variant: row map and rotary table
   int* row_map = reinterpret_cast<int*>(wsb + pl.off_rowmap);
+  int* off_map = reinterpret_cast<int*>(wsb + pl.off_offmap);
   float2* rope_tab = reinterpret_cast<float2*>(wsb + pl.off_tab);
   if (fused != nullptr) {
     FusedPlanParams fp;
     fp.ctx_off = reinterpret_cast<const long long*>(ctx_off);
     fp.sel_idx = fused->sel_idx;
     fp.shot_off = reinterpret_cast<const long long*>(fused->pool->shot_off);
-    fp.row_map = row_map; fp.rope_tab = rope_tab;
+    fp.row_map = row_map; fp.off_map = off_map; fp.rope_tab = rope_tab;
     fp.ctx_cap = ctx_cap; fp.tab_rows = pl.tab_rows;
     fp.B = B; fp.k = k; fp.n_shots = fused->pool->n_shots; fp.half_d = D / 2;
     fp.rope_base = model->rope_base;
@@ -1310,7 +1325,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     ap.v_pool = static_cast<const __nv_bfloat16*>(fused->pool->v);
     ap.kq_rot = kq_rot;
     ap.vq = static_cast<const __nv_bfloat16*>(vq);
-    ap.row_map = row_map; ap.rope_tab = rope_tab;
+    ap.row_map = row_map; ap.off_map = off_map; ap.k_pos_mode = model->k_pos_mode; ap.rope_tab = rope_tab;
     ap.pool_tokens = fused->pool->pool_tokens; ap.ctx_cap = ctx_cap;
     ap.layer_begin = fused->layer_begin; ap.rope_base_f = model->rope_base;
     if (!attr_done[1][D == 128]) {
@@ -1403,7 +1418,7 @@ extern "C" int adapshot_query_attn_fused(const adapshot_model_t* model, const ad
       pool->pool_tokens <= 0)
     return ADAPSHOT_EINVAL;
   if (B <= 0 || k <= 0 || Tq <= 0 || ctx_cap <= 0 || flags != 0) return ADAPSHOT_EINVAL;
-  if (model->dtype != ADAPSHOT_BF16 || model->k_pos_mode != 0) return ADAPSHOT_EUNSUPPORTED;
+  if (model->dtype != ADAPSHOT_BF16 || (model->k_pos_mode != 0 && model->k_pos_mode != 1)) return ADAPSHOT_EUNSUPPORTED;
   if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
   if (!(model->rope_base > 1.0)) return ADAPSHOT_EINVAL;
   if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;

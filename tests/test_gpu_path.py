@@ -11,14 +11,14 @@ from tests import helpers as hp
 pytestmark = pytest.mark.gpu
 
 
-def oracle_path(w, pool, qs, nl, tau):
+def oracle_path(w, pool, qs, nl, tau, k_pos_mode=0):
     """Oracle results for every query of the workload (K' kept in fp64, never rounded)."""
     sel, _ = orc.select_topk(hp.f64(qs["q_emb"]), hp.f64(pool["emb"]), w.k)
     off = orc.plan_offsets(sel, pool["shot_off"])
     kp, vp = hp.f64(pool["k"][:nl]), hp.f64(pool["v"][:nl])
     outs = []
     for b in range(w.batch):
-        kc, vc, _ = orc.assemble_kv(kp, vp, pool["shot_off"], sel[b], w.rope_base)
+        kc, vc, _ = orc.assemble_kv(kp, vp, pool["shot_off"], sel[b], w.rope_base, k_pos_mode)
         L_list = [int(off[b, n]) for n in w.probes]
         per_layer = [orc.query_attn(hp.f64(qs["q"][b, l]), hp.f64(qs["kq"][b, l]), hp.f64(qs["vq"][b, l]),
                                     kc[l], vc[l], L_list, w.rope_base)[0] for l in range(nl)]
@@ -162,3 +162,29 @@ def test_host_buffer_pass_equals_the_device_pass(fused):
             x.zero_()
     graph.replay()
     same()
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_paper_literal_key_store_whole_path(fused):
+    """k_pos_mode 1 (pool K stored rotated at shot-local positions, angle = the shot's offset,
+    Eq. 7 as printed), materialised and fused, against the oracle chain in the same mode."""
+    from paper_2605_03644_b200 import binding as ab
+    from paper_2605_03644_b200.pipeline import ReusePath
+    nl = 2
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=80, batch=2, k=24, probes=(5, 24), t_q=40, vocab=1800, seed=61)
+    pool, qs = wl.make_pool(w, n_layers=nl), wl.make_queries(w, n_layers=nl)
+    tau = 7.0
+    sel, off, out_want, H_want, fo_want = oracle_path(w, pool, qs, nl, tau, k_pos_mode=1)
+    # the mode matters: the same stored values read as position-free keys give another result
+    _, _, out_mode0, _, _ = oracle_path(w, pool, qs, nl, tau, k_pos_mode=0)
+    assert np.abs(out_mode0 - out_want).max() > 0.1
+    dp = hp.dev_pool(ab, pool)
+    model = hp.model_of(ab, w, n_layers=nl, k_pos_mode=1)
+    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, w.k * w.len_hi, 1, fused=fused)
+    chunk = lambda x: [x[:, lb:le].contiguous().cuda() for lb, le in path.chunks]
+    out, H, fo = path.run(qs["q_emb"].cuda(), chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"].cuda(), tau)
+    torch.cuda.synchronize()
+    assert path.status.item() == 0
+    assert np.array_equal(path.sel_idx.cpu().numpy(), sel) and np.array_equal(path.ctx_off.cpu().numpy(), off)
+    err = np.abs(torch.cat(out, dim=1).cpu().double().numpy() - out_want)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
