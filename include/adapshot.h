@@ -126,6 +126,19 @@ ADAPSHOT_API int adapshot_assemble_kv(const adapshot_model_t* model, const adaps
                          int64_t* ctx_off, uint32_t flags,
                          int32_t* status, void* stream);
 
+/* The same for the selected shots shot_begin .. k-1 only: positions from
+ * ctx_off[b][shot_begin] on are written (and the zero fill after L), earlier positions
+ * of k_ctx / v_ctx are left as they are.  Nested probes share their prefix (Sec. 4.1): a
+ * cache assembled for the first shot_begin shots of the same sel_idx is extended in
+ * place, at the cost of the new shots only.  0 <= shot_begin < k; ctx_off is written in
+ * full (unless ADAPSHOT_ASSEMBLE_KEEP_PLAN).  shot_begin = 0 is adapshot_assemble_kv.   */
+ADAPSHOT_API int adapshot_assemble_kv_from(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                              const int32_t* sel_idx, int32_t B, int32_t k, int32_t shot_begin,
+                              int32_t layer_begin, int32_t layer_end,
+                              void* k_ctx, void* v_ctx, int64_t ctx_cap,
+                              int64_t* ctx_off, uint32_t flags,
+                              int32_t* status, void* stream);
+
 /* ---- Step 3: probe attention over the reused cache (Eq. 1; tree mask of
  * Sec. 4.1: probe j sees the first probe_nshots[j] shots, i.e. context tokens
  * 0 .. L_j-1 with L_j = ctx_off[b][probe_nshots[j]], and causally its own T_q

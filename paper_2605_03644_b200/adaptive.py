@@ -3,8 +3,8 @@ shot counts n0, n0 + step, ... ; the answer is the smallest shot count whose las
 entropy (Eq. 2) is at most tau, and probing stops with the round that finds it.
 
 The driver only sequences the C-ABI steps and keeps the books: selection once for the
-largest shot count, then per round the gather of the round's longest prefix (nested
-prefixes share their re-encoded positions, so earlier shots land where they were), the
+largest shot count, then per round the gather of the shots the round adds (nested
+prefixes share their re-encoded positions, so the earlier shots stay where they are), the
 probe attention of the round's m probes over it and the entropy rule on the logits the
 caller's model produced for those probes.  It does no arithmetic on tensors itself.
 """
@@ -67,15 +67,18 @@ class ProbeRounds:
         return self._ctx_off[: self.B * (k + 1)].view(self.B, k + 1)
 
     def run_round(self, r: int, q, kq, vq, logits, tau: float):
-        """Gather the prefix of round r's largest probe, attend with its m probes, apply the
-        entropy rule to `logits` ([B*m][V], the model's last-token logits of those probes)."""
+        """Extend the cache to round r's largest probe (rounds must be run in order, from 0),
+        attend with its m probes, apply the entropy rule to `logits` ([B*m][V], the model's
+        last-token logits of those probes)."""
         probes = self.schedule[r]
         k_r = probes[-1]
         nl = self.model.n_layers
         sel_r = self.sel_idx[:, :k_r].contiguous()
         off_r = self.ctx_off(k_r)
-        ab.adapshot_assemble_kv(self.model, self.pool, sel_r, 0, nl, self.k_ctx, self.v_ctx, self.ctx_cap,
-                                off_r, self.status)
+        # the earlier rounds' shots are in place already: only the new ones are gathered
+        first_new = self.schedule[r - 1][-1] if r > 0 else 0
+        ab.adapshot_assemble_kv_from(self.model, self.pool, sel_r, first_new, 0, nl, self.k_ctx, self.v_ctx,
+                                     self.ctx_cap, off_r, self.status)
         ab.adapshot_query_attn(self.model, self.k_ctx, self.v_ctx, self.ctx_cap, off_r, k_r, probes,
                                q, kq, vq, 0, nl, self.out, None, self.ws_attn, self.status)
         ab.adapshot_entropy(logits, self.H, tau, self.m, self.first_ok, self.ws_entropy, self.status)

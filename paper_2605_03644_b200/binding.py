@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 ASSEMBLE_KEEP_PLAN = 1
 
 EXPORTS = [
-    "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv",
+    "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv", "adapshot_assemble_kv_from",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_subset",
@@ -59,6 +59,9 @@ _select = _sig("adapshot_select", C.c_int, [C.POINTER(PoolT), _vp, _i32, _i32, _
 _assemble = _sig("adapshot_assemble_kv", C.c_int,
                  [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _i32, _i32, _i32, _i32, _vp, _vp, _i64,
                   _vp, _u32, _vp, _vp])
+_assemble_from = _sig("adapshot_assemble_kv_from", C.c_int,
+                      [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _i64,
+                       _vp, _u32, _vp, _vp])
 _entropy_ws = _sig("adapshot_entropy_workspace_bytes", _sz, [_i32, _i32])
 _entropy = _sig("adapshot_entropy", C.c_int,
                 [_vp, _i32, _i32, _i32, _i64, _vp, _f, _i32, _vp, _vp, _sz, _vp, _vp])
@@ -167,6 +170,15 @@ def adapshot_assemble_kv(model: ModelT, pool: Pool, sel_idx: torch.Tensor, layer
     B, k = sel_idx.shape
     _check(_assemble(C.byref(model), C.byref(pool.c), _ptr(sel_idx), B, k, layer_begin, layer_end,
                      _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), flags, _ptr(status), _stream()))
+
+
+def adapshot_assemble_kv_from(model: ModelT, pool: Pool, sel_idx: torch.Tensor, shot_begin: int,
+                              layer_begin: int, layer_end: int, k_ctx: torch.Tensor, v_ctx: torch.Tensor,
+                              ctx_cap: int, ctx_off: torch.Tensor, status: torch.Tensor, flags: int = 0):
+    B, k = sel_idx.shape
+    _check(_assemble_from(C.byref(model), C.byref(pool.c), _ptr(sel_idx), B, k, shot_begin, layer_begin,
+                          layer_end, _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), flags, _ptr(status),
+                          _stream()))
 
 
 def adapshot_attn_workspace_bytes(model: ModelT, B: int, P: int, Tq: int, n_layers_in_call: int,

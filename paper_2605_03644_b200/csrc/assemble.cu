@@ -104,6 +104,7 @@ struct GatherArgs {
   long long ctx_cap;
   int n_shots, B, k, n_kv_heads;
   int layer_begin, n_layers_call;
+  int shot_begin;              // first selected shot to gather (earlier positions of the cache are kept)
   int k_pos_mode;
   double rope_base;
   int32_t* status;
@@ -155,7 +156,8 @@ gather_rope_kernel(const GatherArgs a) {
     const long long* off = a.ctx_off + (long long)b * (a.k + 1);
     const long long L = off[a.k];
     const long long pad_end = (L + kTile - 1) / kTile * kTile;
-    if (p0 >= pad_end) continue;
+    const long long first_pos = off[a.shot_begin];                // positions before it stay as they are
+    if (p0 >= pad_end || p0 + kRun <= first_pos) continue;
     int lo = 0;
     long long o = 0, o_next = 0, src0 = 0;
     int s = -1;
@@ -181,6 +183,7 @@ gather_rope_kernel(const GatherArgs a) {
     for (int tt = 0; tt < kRun; ++tt) {
     const long long p = p0 + tt;
     if (p >= a.ctx_cap) break;
+    if (p < first_pos) continue;
     if (p >= L) {
       // zero the rest of the last 128-token tile so whole tiles can be read later
       if (p < pad_end) {
@@ -292,7 +295,17 @@ extern "C" int adapshot_assemble_kv(const adapshot_model_t* model, const adapsho
                                     int32_t layer_begin, int32_t layer_end, void* k_ctx, void* v_ctx,
                                     int64_t ctx_cap, int64_t* ctx_off, uint32_t flags,
                                     int32_t* status, void* stream) {
+  return adapshot_assemble_kv_from(model, pool, sel_idx, B, k, 0, layer_begin, layer_end, k_ctx, v_ctx, ctx_cap,
+                                   ctx_off, flags, status, stream);
+}
+
+extern "C" int adapshot_assemble_kv_from(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                                         const int32_t* sel_idx, int32_t B, int32_t k, int32_t shot_begin,
+                                         int32_t layer_begin, int32_t layer_end, void* k_ctx, void* v_ctx,
+                                         int64_t ctx_cap, int64_t* ctx_off, uint32_t flags,
+                                         int32_t* status, void* stream) {
   if (model == nullptr || pool == nullptr || sel_idx == nullptr || ctx_off == nullptr) return ADAPSHOT_EINVAL;
+  if (shot_begin < 0 || shot_begin >= k) return ADAPSHOT_ESHAPE;
   if (B <= 0 || (flags & ~ADAPSHOT_ASSEMBLE_KEEP_PLAN) != 0 || pool->shot_off == nullptr || pool->n_shots <= 0)
     return ADAPSHOT_EINVAL;
   if (k < 1 || k > pool->n_shots) return ADAPSHOT_ESHAPE;
@@ -332,6 +345,7 @@ extern "C" int adapshot_assemble_kv(const adapshot_model_t* model, const adapsho
   a.pool_tokens = pool->pool_tokens; a.ctx_cap = ctx_cap;
   a.n_shots = pool->n_shots; a.B = B; a.k = k; a.n_kv_heads = model->n_kv_heads;
   a.layer_begin = layer_begin; a.n_layers_call = layer_end - layer_begin;
+  a.shot_begin = shot_begin;
   a.k_pos_mode = model->k_pos_mode; a.rope_base = model->rope_base; a.status = status;
   for (int i = 0; i < model->head_dim / 2; ++i)
     a.theta[i] = pow(model->rope_base, -2.0 * (double)i / (double)model->head_dim);

@@ -69,6 +69,10 @@ def test_host_side_argument_checks_launch_nothing(ab):
     assert asm(*args(bad)) == ab.ESHAPE                               # head_dim not 64 / 128
     bad = ab.make_model(1, 5, 2, 64, "fp32", 1e4)
     assert asm(*args(bad)) == ab.ESHAPE                               # Hq % Hkv != 0
+    asm_from = ab.lib.adapshot_assemble_kv_from
+    from_args = lambda sb: [C.byref(model), C.byref(pool), fake, 1, 4, sb, 0, 1, fake, fake, 256, fake, 0, None, None]
+    assert asm_from(*from_args(4)) == ab.ESHAPE                       # shot_begin must be < k
+    assert asm_from(*from_args(-1)) == ab.ESHAPE
     ent = ab.lib.adapshot_entropy
     assert ent(None, 0, 1, 8, 8, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EINVAL
     assert ent(fake, 2, 1, 8, 8, fake, 0.5, 1, None, fake, 1 << 20, None, None) == ab.EUNSUPPORTED

@@ -119,3 +119,39 @@ def test_plan_only_capacity_and_bad_ids():
     kc, vc, off, st = hp.run_assemble(ab, model, dp, bad, 128, 0, 1, torch.float32)
     assert st == ab.EINDEX and off.tolist() == [[0, 32, 32, 64]]
     assert torch.equal(vc[0, 0, 32:64], pool["v"][0, 64:96].cuda())
+
+
+@pytest.mark.parametrize("k_pos_mode", [0, 1])
+def test_extending_a_nested_prefix_equals_one_gather(k_pos_mode):
+    """adapshot_assemble_kv_from: a cache assembled for the first k1 shots and extended with
+    shots k1 .. k2-1 is, bit for bit, the cache assembled for k2 shots at once (K, V, the zero
+    fill and the untouched canary), and the extension leaves the first positions alone."""
+    ab = hp.gpu_binding()
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=60, batch=3, k=20, probes=(20,), seed=71)
+    nl = 3
+    pool = wl.make_pool(w, n_layers=nl)
+    dp = hp.dev_pool(ab, pool)
+    rng = np.random.default_rng(71)
+    sel_np = np.stack([rng.permutation(w.n_shots)[:w.k] for _ in range(w.batch)]).astype(np.int32)
+    sel = torch.from_numpy(sel_np).cuda()
+    model = hp.model_of(ab, w, n_layers=nl, k_pos_mode=k_pos_mode)
+    cap = w.k * w.len_hi
+    want_k, want_v, want_off, st = hp.run_assemble(ab, model, dp, sel, cap, 0, nl, torch.bfloat16)
+    assert st == 0
+    for k1 in (1, 7, 19):
+        sel1 = sel[:, :k1].contiguous()
+        kc, vc, off1, st = hp.run_assemble(ab, model, dp, sel1, cap, 0, nl, torch.bfloat16)
+        assert st == 0
+        # poison the first positions: the extension must not rewrite them
+        first = off1[:, k1].cpu().numpy()
+        keep_k, keep_v = kc.clone(), vc.clone()
+        off2 = torch.full((w.batch, w.k + 1), -1, dtype=torch.int64, device="cuda")
+        status = hp.new_status()
+        ab.adapshot_assemble_kv_from(model, dp, sel, k1, 0, nl, kc, vc, cap, off2, status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert torch.equal(off2, want_off)
+        assert torch.equal(kc, want_k) and torch.equal(vc, want_v)
+        for b in range(w.batch):
+            assert torch.equal(kc[b, :, :first[b]], keep_k[b, :, :first[b]])
+            assert torch.equal(vc[b, :, :first[b]], keep_v[b, :, :first[b]])
