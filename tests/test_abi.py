@@ -69,6 +69,15 @@ def test_host_side_argument_checks_launch_nothing(ab):
     assert asm(*args(bad)) == ab.ESHAPE                               # head_dim not 64 / 128
     bad = ab.make_model(1, 5, 2, 64, "fp32", 1e4)
     assert asm(*args(bad)) == ab.ESHAPE                               # Hq % Hkv != 0
+    # attention: more (probe, query) pairs than one call takes, probes not ascending
+    amodel = ab.make_model(1, 4, 1, 64, "bf16", 1e4)
+    att = ab.lib.adapshot_query_attn
+    probes = (C.c_int32 * 4)(1, 2, 3, 4)
+    att_args = lambda B, pr, P: [C.byref(amodel), fake, fake, 256, fake, B, 4, pr, P, fake, fake, fake, 8, 0, 1,
+                                 fake, None, 0, C.c_void_p(0x1000), 1 << 40, None, None]
+    assert att(*att_args(65, probes, 4)) == ab.ESHAPE                  # 65 * 4 > 256 pairs
+    assert att(*att_args(1, (C.c_int32 * 2)(3, 3), 2)) == ab.ESHAPE    # not strictly ascending
+    assert att(*att_args(1, (C.c_int32 * 1)(5), 1)) == ab.ESHAPE       # more shots than k
     asm_from = ab.lib.adapshot_assemble_kv_from
     from_args = lambda sb: [C.byref(model), C.byref(pool), fake, 1, 4, sb, 0, 1, fake, fake, 256, fake, 0, None, None]
     assert asm_from(*from_args(4)) == ab.ESHAPE                       # shot_begin must be < k

@@ -108,3 +108,12 @@ def test_head_dim_64_bf16_many_tiles():
                                   n_q_heads=6, n_kv_heads=3, seed=24)
     sel = np.random.default_rng(2).permutation(32)[:20].astype(np.int32)[None]
     _run_case(w, sel, [20], 1)
+
+
+def test_maximum_number_of_probe_query_pairs():
+    # B * P = 256 (the most one call takes): 64 queries x 4 nested probes, short shots, G = 8
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=40, len_lo=20, len_hi=60, batch=64, k=6, t_q=5, n_q_heads=8,
+                                  n_kv_heads=1, seed=25, channel_scale=False)
+    rng = np.random.default_rng(3)
+    sel = np.stack([rng.permutation(40)[:6] for _ in range(64)]).astype(np.int32)
+    _run_case(w, sel, [1, 2, 4, 6], 1)
