@@ -92,7 +92,10 @@ typedef struct adapshot_pool {
  * sel_idx[b][r] = id of the r-th most relevant shot, equal scores ordered by
  * the lower id.  Nested probes use prefixes of sel_idx.
  *   q_emb [B][emb_dim] fp32; sel_idx [B][k] int32 out; sel_score [B][k] fp32 out
- *   or NULL.  Needs 1 <= k <= n_shots.  Scores are compared in fp64.            */
+ *   or NULL.  Needs 1 <= k <= n_shots (else ADAPSHOT_ESHAPE); a pool of more than
+ *   8192 shots (one sort chunk) takes k <= 4096 (else ADAPSHOT_EUNSUPPORTED: the
+ *   chunks' candidate lists would not shrink from one merge round to the next).
+ *   Scores are compared in fp64.                                                */
 ADAPSHOT_API size_t adapshot_select_workspace_bytes(int32_t n_shots, int32_t B, int32_t k);
 ADAPSHOT_API int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, int32_t B, int32_t k,
                     int32_t* sel_idx, float* sel_score,
@@ -152,9 +155,15 @@ ADAPSHOT_API int adapshot_assemble_kv_from(const adapshot_model_t* model, const 
  *         log-sum-exp of the scaled scores, or NULL
  *   probe_nshots : HOST int32 [P], strictly ascending, 1 <= n_j <= k
  *   k_ctx, v_ctx, ctx_cap, ctx_off: as written by adapshot_assemble_kv for the
- *   same B, k and layer range (ctx_cap a multiple of 8).
+ *   same B, k and layer range.
  * bf16 tensor-core kernel (tcgen05, fp32 accumulation, split over the context
- * with a log-sum-exp merge); model->dtype must be ADAPSHOT_BF16.                */
+ * with a log-sum-exp merge); model->dtype must be ADAPSHOT_BF16.
+ * Limits of one call (ADAPSHOT_ESHAPE beyond them, nothing launched): P <= 16
+ * probes, B * P <= 256 (probe, query) pairs, ctx_cap < 2^31 - 256.
+ * Every wait inside the kernel is bounded by about two seconds of SM clock; a GPU
+ * that is time-sliced with other work for longer than that in the middle of a
+ * call can therefore report a spurious ADAPSHOT_ETIMEOUT in `status` (the
+ * outputs of that call are then incomplete: repeat it).                         */
 ADAPSHOT_API size_t adapshot_attn_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
                                      int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap);
 ADAPSHOT_API int adapshot_query_attn(const adapshot_model_t* model,
@@ -193,7 +202,10 @@ ADAPSHOT_API int adapshot_query_attn_fused(const adapshot_model_t* model, const 
  *   first_ok[g] = smallest j in 0..rows_per_group-1 with
  *                 H[g*rows_per_group + j] <= tau, else -1   (int32 out, or NULL)
  *   logits [R][row_stride] fp32 or bf16 (dtype), row_stride in elements, rows
- *   16-byte aligned; one pass with a running maximum, fp32 accumulation.        */
+ *   16-byte aligned; one pass with a running maximum, fp32 accumulation.
+ *   Limits: R a multiple of rows_per_group, rows_per_group <= 8192, and
+ *   R * splits < 2^31 with splits = min(ceil(296 / R), ceil(V / 4096)) (one CTA
+ *   per row and split); ADAPSHOT_ESHAPE otherwise.                              */
 ADAPSHOT_API size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V);
 ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V, int64_t row_stride,
                      float* H, float tau, int32_t rows_per_group, int32_t* first_ok,

@@ -274,7 +274,9 @@ int launch_gather(GatherArgs a, cudaStream_t st) {
   // Resident warps: about six 128-thread CTAs per SM.  Long runs amortise the plan lookup; a
   // small launch takes shorter runs so that every resident warp gets several and the tail
   // wave stays short.
-  const long long resident_warps = 148ll * 6 * warps_per_block;
+  const long long n_sm = ads_sm_count();
+  if (n_sm <= 0) return ADAPSHOT_ECUDA;
+  const long long resident_warps = n_sm * 6 * warps_per_block;
   const long long tokens = (long long)a.B * a.ctx_cap;
   a.run = kRunMax;
   while (a.run > 1 && tokens / a.run < 4 * resident_warps) a.run >>= 1;
@@ -282,7 +284,7 @@ int launch_gather(GatherArgs a, cudaStream_t st) {
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
   // measured: one resident wave with a grid-stride loop is best when a run is short (one
   // layer per call), several waves when every run walks several layers
-  const long long max_blocks = a.n_layers_call == 1 ? 148ll * 6 : 148ll * 16 * 4;
+  const long long max_blocks = a.n_layers_call == 1 ? n_sm * 6 : n_sm * 16 * 4;
   if (blocks > max_blocks) blocks = max_blocks;
   gather_rope_kernel<T, D><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
   return ads_launch_status();

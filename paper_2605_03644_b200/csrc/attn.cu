@@ -1231,12 +1231,8 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   float* o_part = reinterpret_cast<float*>(wsb + pl.off_opart);
   float* ml_part = reinterpret_cast<float*>(wsb + pl.off_ml);
 
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    ADS_CHECK_CUDA(cudaGetDevice(&dev));
-    ADS_CHECK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-  }
+  const int n_sm = ads_sm_count();
+  if (n_sm <= 0) return ADAPSHOT_ECUDA;
   const int n_cta = n_sm < kMaxCtas ? n_sm : kMaxCtas;
   const int n_gangs = n_cta / pl.gang > 0 ? n_cta / pl.gang : 1;
 
@@ -1283,7 +1279,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     fp.rope_base = model->rope_base;
     const long long work = (long long)B * ctx_cap + pl.tab_rows * (D / 2);
     long long blocks = (work + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > n_sm * 16) blocks = n_sm * 16;
     attn_fused_plan_kernel<<<(unsigned)blocks, 256, 0, st>>>(fp);
     if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   }
@@ -1310,14 +1306,10 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
   const int smem = (int)AttnSmem<128, false>::kTotal;     // same request for D = 64 and for the fused variant: one CTA per SM
-  static bool attr_done[2][2] = {{false, false}, {false, false}};
+  static bool attr_done[2][kAdsMaxDevices] = {{false}, {false}};   // per template instance (D) and device
   if (g_profile) ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[0], st));
   if (fused == nullptr) {
-    if (!attr_done[0][D == 128]) {
-      ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          smem));
-      attr_done[0][D == 128] = true;
-    }
+    if (ads_set_max_smem(attn_main_kernel<D, false>, smem, attr_done[0]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
     attn_main_kernel<D, false><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(
         tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   } else {
@@ -1328,11 +1320,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     ap.row_map = row_map; ap.off_map = off_map; ap.k_pos_mode = model->k_pos_mode; ap.rope_tab = rope_tab;
     ap.pool_tokens = fused->pool->pool_tokens; ap.ctx_cap = ctx_cap;
     ap.layer_begin = fused->layer_begin; ap.rope_base_f = model->rope_base;
-    if (!attr_done[1][D == 128]) {
-      ADS_CHECK_CUDA(cudaFuncSetAttribute(attn_main_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          smem));
-      attr_done[1][D == 128] = true;
-    }
+    if (ads_set_max_smem(attn_main_kernel<D, true>, smem, attr_done[1]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
     attn_main_kernel<D, true><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
         tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   }

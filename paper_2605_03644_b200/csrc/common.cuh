@@ -23,6 +23,40 @@ static inline int ads_launch_status() {
   return cudaGetLastError() == cudaSuccess ? ADAPSHOT_OK : ADAPSHOT_ECUDA;
 }
 
+// Per-device host-side caches: a process may drive several GPUs, and both the SM count and a
+// kernel's shared-memory attribute belong to the device that is current at the call.
+constexpr int kAdsMaxDevices = 64;
+static inline int ads_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kAdsMaxDevices) return -1;
+  return dev;
+}
+// SM count of the current device (0 on error); looked up once per device.
+static inline int ads_sm_count() {
+  static int n_sm[kAdsMaxDevices] = {0};
+  const int dev = ads_current_device();
+  if (dev < 0) return 0;
+  if (n_sm[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 0;
+    n_sm[dev] = n;
+  }
+  return n_sm[dev];
+}
+// Raises a kernel's dynamic shared-memory limit once per device.  `done` is a per-kernel table
+// (kAdsMaxDevices entries) owned by the caller.  The value is the same every time, so two
+// threads that race here both write it.
+template <typename Kernel>
+static inline int ads_set_max_smem(Kernel kernel, int bytes, bool* done) {
+  const int dev = ads_current_device();
+  if (dev < 0) return ADAPSHOT_ECUDA;
+  if (!done[dev]) {
+    ADS_CHECK_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done[dev] = true;
+  }
+  return ADAPSHOT_OK;
+}
+
 // Device: record an error code once; later codes do not overwrite the first.
 __device__ __forceinline__ void ads_set_status(int32_t* status, int32_t code) {
   if (status != nullptr) atomicCAS(status, 0, code);

@@ -63,13 +63,15 @@ __device__ __forceinline__ EntState ent_warp_reduce(EntState st) {
 
 constexpr int kEntThreads = 256;
 
-// grid (n_split, R).  partial[(r * n_split + s)] = state of slice s of row r.
+// One-dimensional grid of R * n_split blocks (block = r * n_split + s, so the row count is not
+// bound by the 65535 limit of the other grid dimensions).
+// partial[(r * n_split + s)] = state of slice s of row r.
 template <typename T>
 __global__ void __launch_bounds__(kEntThreads)
-entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride, int slice,
+entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride, int slice, int n_split,
                        float* __restrict__ partial) {
   constexpr int kVec = 16 / sizeof(T);
-  const int r = blockIdx.y, sp = blockIdx.x, n_split = gridDim.x;
+  const int r = blockIdx.x / n_split, sp = blockIdx.x % n_split;
   const T* row = logits + (long long)r * row_stride;
   const int begin = sp * slice;
   const int end = min(V, begin + slice);
@@ -208,9 +210,13 @@ entropy_subset_finish_kernel(const float* __restrict__ partial, int n_split, int
   }
 }
 
+// A fixed figure rather than the SM count of the current device, so that the workspace size
+// can be asked for without a device and does not change from one GPU to another.
+constexpr int kEntTargetCtas = 296;
+
 int ent_splits(int R, int V) {
-  // enough CTAs for about two waves of 148 SMs, each slice at least 4096 entries
-  int want = (2 * 148 + R - 1) / R;
+  // about kEntTargetCtas CTAs in all, each slice at least 4096 entries
+  int want = (kEntTargetCtas + R - 1) / R;
   int max_by_len = (V + 4095) / 4096;
   int s = want < max_by_len ? want : max_by_len;
   return s < 1 ? 1 : s;
@@ -233,6 +239,7 @@ extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, in
   if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
   if (rows_per_group <= 0) rows_per_group = 1;
   if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  if ((long long)R * ent_splits(R, V) > 0x7fffffffll) return ADAPSHOT_ESHAPE;
   const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
   if (!ads_aligned16(logits) || !ads_aligned16(ws) || (row_stride * es) % 16 != 0) return ADAPSHOT_EALIGN;
   if (ws_bytes < adapshot_entropy_workspace_bytes(R, V)) return ADAPSHOT_ECAPACITY;
@@ -242,14 +249,14 @@ extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, in
   const int vec = 16 / (int)es;
   int slice = (V + n_split - 1) / n_split;
   slice = (slice + vec - 1) / vec * vec;
-  dim3 grid(n_split, R);
+  const unsigned grid = (unsigned)((long long)R * n_split);
   float* partial = static_cast<float*>(ws);
   if (dtype == ADAPSHOT_F32)
     entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(
-        static_cast<const float*>(logits), V, row_stride, slice, partial);
+        static_cast<const float*>(logits), V, row_stride, slice, n_split, partial);
   else
     entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, partial);
+        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, n_split, partial);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   entropy_finish_kernel<<<R / rows_per_group, 256, rows_per_group * sizeof(float), st>>>(
       partial, n_split, R, rows_per_group, tau, H, first_ok);
@@ -268,6 +275,7 @@ extern "C" int adapshot_entropy_subset(const void* logits, int32_t dtype, int32_
   if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
   if (rows_per_group <= 0) rows_per_group = 1;
   if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  if ((long long)R * ent_splits(R, V) > 0x7fffffffll) return ADAPSHOT_ESHAPE;
   const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
   if (!ads_aligned16(logits) || !ads_aligned16(ws) || (row_stride * es) % 16 != 0 ||
       ((uintptr_t)subset_ids & 3u))
@@ -279,20 +287,20 @@ extern "C" int adapshot_entropy_subset(const void* logits, int32_t dtype, int32_
   const int vec = 16 / (int)es;
   int slice = (V + n_split - 1) / n_split;
   slice = (slice + vec - 1) / vec * vec;
-  dim3 grid(n_split, R);
+  const unsigned grid = (unsigned)((long long)R * n_split);
   float* partial = static_cast<float*>(ws);
   const int renorm = (int)(flags & 1u);
   const size_t sh = rows_per_group * sizeof(float);
   if (dtype == ADAPSHOT_F32) {
     const float* lg = static_cast<const float*>(logits);
-    entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, partial);
+    entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, n_split, partial);
     if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
     entropy_subset_finish_kernel<float><<<R / rows_per_group, 256, sh, st>>>(
         partial, n_split, R, rows_per_group, lg, row_stride, V, subset_ids, n_subset, renorm, tau, H, first_ok,
         status);
   } else {
     const __nv_bfloat16* lg = static_cast<const __nv_bfloat16*>(logits);
-    entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, partial);
+    entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(lg, V, row_stride, slice, n_split, partial);
     if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
     entropy_subset_finish_kernel<__nv_bfloat16><<<R / rows_per_group, 256, sh, st>>>(
         partial, n_split, R, rows_per_group, lg, row_stride, V, subset_ids, n_subset, renorm, tau, H, first_ok,
@@ -344,6 +352,7 @@ extern "C" int adapshot_entropy_static(const void* logits, int32_t dtype, int32_
   if (dtype != ADAPSHOT_F32 && dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
   if (rows_per_group <= 0) rows_per_group = 1;
   if (R % rows_per_group != 0 || rows_per_group > 8192) return ADAPSHOT_ESHAPE;
+  if ((long long)R * ent_splits(R, V) > 0x7fffffffll) return ADAPSHOT_ESHAPE;
   const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
   if (!ads_aligned16(logits) || (row_stride * es) % 16 != 0) return ADAPSHOT_EALIGN;
   const int n_split = ent_splits(R, V);
@@ -357,15 +366,15 @@ extern "C" int adapshot_entropy_static(const void* logits, int32_t dtype, int32_
   const int vec = 16 / (int)es;
   int slice = (V + n_split - 1) / n_split;
   slice = (slice + vec - 1) / vec * vec;
-  dim3 grid(n_split, R);
+  const unsigned grid = (unsigned)((long long)R * n_split);
   // every (row, split) state this call reads is written by the first kernel, so
   // nothing in the shared array has to start at zero
   if (dtype == ADAPSHOT_F32)
     entropy_partial_kernel<float><<<grid, kEntThreads, 0, st>>>(
-        static_cast<const float*>(logits), V, row_stride, slice, partial);
+        static_cast<const float*>(logits), V, row_stride, slice, n_split, partial);
   else
     entropy_partial_kernel<__nv_bfloat16><<<grid, kEntThreads, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, partial);
+        static_cast<const __nv_bfloat16*>(logits), V, row_stride, slice, n_split, partial);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   entropy_finish_kernel<<<R / rows_per_group, 256, rows_per_group * sizeof(float), st>>>(
       partial, n_split, R, rows_per_group, tau, H, first_ok);

@@ -282,11 +282,8 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
   }
 
   const size_t smem = (size_t)kSortCap * (8 + 4);
-  static bool attr_set = false;   // same value every time: a benign race
-  if (!attr_set) {
-    ADS_CHECK_CUDA(cudaFuncSetAttribute(topk_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_set = true;
-  }
+  static bool attr_set[kAdsMaxDevices] = {false};
+  if (ads_set_max_smem(topk_sort_kernel, (int)smem, attr_set) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   int n_in = N, in_stride = N;
   int round = 0;

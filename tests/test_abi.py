@@ -57,6 +57,10 @@ def test_host_side_argument_checks_launch_nothing(ab):
     assert sel(C.byref(pool), fake, 1, 0, fake, None, fake, 1 << 20, None, None) == ab.ESHAPE
     assert sel(C.byref(pool), C.c_void_p(0x1004), 1, 4, fake, None, fake, 1 << 20, None, None) == ab.EALIGN
     assert sel(C.byref(pool), fake, 1, 4, fake, None, fake, 16, None, None) == ab.ECAPACITY
+    # pools beyond one sort chunk (8192 shots) take at most 4096 shots per query
+    big = ab.PoolT(9000, 8, 100, 0x1000, 0x1000, 0x1000, 0x1000)
+    assert sel(C.byref(big), fake, 1, 4097, fake, None, fake, 1 << 30, None, None) == ab.EUNSUPPORTED
+    assert sel(C.byref(big), fake, 1, 4096, fake, None, fake, 16, None, None) == ab.ECAPACITY      # accepted shape
     asm = ab.lib.adapshot_assemble_kv
     args = lambda m, **kw: [C.byref(m), C.byref(pool), fake, 1, kw.get("k", 4), kw.get("lb", 0), kw.get("le", 1),
                             kw.get("kc", fake), kw.get("vc", fake), kw.get("cap", 256), fake, kw.get("flags", 0), None, None]
@@ -76,6 +80,7 @@ def test_host_side_argument_checks_launch_nothing(ab):
     att_args = lambda B, pr, P: [C.byref(amodel), fake, fake, 256, fake, B, 4, pr, P, fake, fake, fake, 8, 0, 1,
                                  fake, None, 0, C.c_void_p(0x1000), 1 << 40, None, None]
     assert att(*att_args(65, probes, 4)) == ab.ESHAPE                  # 65 * 4 > 256 pairs
+    assert att(*att_args(1, (C.c_int32 * 17)(*range(1, 18)), 17)) == ab.ESHAPE   # more than 16 probes
     assert att(*att_args(1, (C.c_int32 * 2)(3, 3), 2)) == ab.ESHAPE    # not strictly ascending
     assert att(*att_args(1, (C.c_int32 * 1)(5), 1)) == ab.ESHAPE       # more shots than k
     asm_from = ab.lib.adapshot_assemble_kv_from

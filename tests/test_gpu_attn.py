@@ -1,7 +1,7 @@
 """adapshot_query_attn vs the fp64 oracle: bf16 output within max-abs 2e-2 and
-mean-abs 2e-3 (the stated tolerance).  The log-sum-exp output has no stated bound:
-it inherits the score error of rounding the rotated q and own k to bf16 (2^-9
-relative per element, a few 1e-3 on scores of magnitude ~1-4), so 1e-2 is used."""
+mean-abs 2e-3 (the stated tolerance, plus the bf16 result's own rounding where a short
+context makes the outputs larger than one; tests.helpers states both bounds and the one
+used for the log-sum-exp output)."""
 import numpy as np
 import pytest
 import torch
@@ -11,7 +11,6 @@ from paper_2605_03644_b200 import workloads as wl
 from tests import helpers as hp
 
 pytestmark = pytest.mark.gpu
-MAX_ABS, MEAN_ABS, LSE_ABS = 2e-2, 2e-3, 1e-2
 
 
 def _oracle_ctx(w, pool, sel_np, nl):
@@ -59,19 +58,16 @@ def _run_case(w, sel_np, probes, nl, cap_extra=37, k_gain=1.0):
                            out, lse, ws, st)
     torch.cuda.synchronize()
     assert st.item() == 0
-    worst, mean_acc, n = 0.0, 0.0, 0
+    got_all, want_all = [], []
     for b in range(B):
         L_list = [int(off[b, n_j]) for n_j in probes]
         for l in range(nl):
             want, want_lse = orc.query_attn(hp.f64(qs["q"][b, l]), hp.f64(qs["kq"][b, l]), hp.f64(qs["vq"][b, l]),
                                             hp.f64(kc[b, l]), hp.f64(vc[b, l]), L_list, w.rope_base)
-            err = np.abs(out[b, l].cpu().double().numpy() - want)
-            worst = max(worst, err.max()); mean_acc += err.sum(); n += err.size
-            # (the score error behind the LSE bound is proportional to the keys' magnitude)
-            assert np.abs(lse[b, l].cpu().double().numpy() - want_lse).max() <= LSE_ABS * k_gain
-    assert worst <= MAX_ABS, worst
-    assert mean_acc / n <= MEAN_ABS, mean_acc / n
-    return worst, mean_acc / n
+            got_all.append(out[b, l].cpu().double().numpy())
+            want_all.append(want)
+            assert np.abs(lse[b, l].cpu().double().numpy() - want_lse).max() <= hp.lse_bound(k_gain)
+    hp.assert_attn_close(np.stack(got_all), np.stack(want_all))
 
 
 def test_cfg1_attention():
@@ -93,8 +89,6 @@ def test_8b_shape_ragged_probes_and_cut_units():
 
 def test_tq_longer_than_a_key_tile_and_g8():
     # T_q = 150 > 128: two own-key tiles with the causal diagonal; G = 8 rows per token
-    # (contexts of a few hundred tokens keep |out| near 1, where the absolute bf16 tolerance applies:
-    # half a bf16 step of an output of magnitude 4 is already 1.6e-2)
     w = wl.CONFIGS["cfg4"].scaled(n_shots=20, len_lo=40, len_hi=70, batch=1, k=9, t_q=150, n_q_heads=16,
                                   n_kv_heads=2, pool_token_target=0, seed=22)
     sel = np.arange(9, dtype=np.int32)[None, ::-1].copy()
@@ -102,8 +96,8 @@ def test_tq_longer_than_a_key_tile_and_g8():
 
 
 def test_single_token_probe_and_tiny_context():
-    # one probe token over 2-6 context tokens; unit-scale V keeps the outputs in the tolerance's range
-    w = wl.CONFIGS["cfg2"].scaled(n_shots=8, len_lo=1, len_hi=3, batch=1, k=2, t_q=1, seed=23, channel_scale=False)
+    # one probe token over 2-6 context tokens
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=8, len_lo=1, len_hi=3, batch=1, k=2, t_q=1, seed=23)
     _run_case(w, np.array([[5, 1]], dtype=np.int32), [1, 2], 1)
 
 
@@ -117,7 +111,7 @@ def test_head_dim_64_bf16_many_tiles():
 def test_maximum_number_of_probe_query_pairs():
     # B * P = 256 (the most one call takes): 64 queries x 4 nested probes, short shots, G = 8
     w = wl.CONFIGS["cfg2"].scaled(n_shots=40, len_lo=20, len_hi=60, batch=64, k=6, t_q=5, n_q_heads=8,
-                                  n_kv_heads=1, seed=25, channel_scale=False)
+                                  n_kv_heads=1, seed=25)
     rng = np.random.default_rng(3)
     sel = np.stack([rng.permutation(40)[:6] for _ in range(64)]).astype(np.int32)
     _run_case(w, sel, [1, 2, 4, 6], 1)
@@ -126,8 +120,54 @@ def test_maximum_number_of_probe_query_pairs():
 def test_peaked_scores_rescale_the_accumulator():
     # keys three times larger: scores of a row spread over tens of log2 units, so the row maximum
     # grows by more than the lazy-rescale threshold several times along the context and the
-    # output approaches single value rows (unit-scale V keeps it in the tolerance's range)
+    # output approaches single value rows.  The factor 3 takes the place of the per-channel scale here
+    # (both together would push the keys six times beyond the configurations' magnitude, and the
+    # score error of the bf16 query with them).
     w = wl.CONFIGS["cfg2"].scaled(n_shots=48, len_lo=60, len_hi=140, batch=1, k=30, t_q=24, seed=26,
                                   channel_scale=False)
     sel = np.random.default_rng(4).permutation(48)[:30].astype(np.int32)[None]
     _run_case(w, sel, [7, 30], 1, k_gain=3.0)
+
+
+def test_a_range_that_spans_more_pairs_than_the_schedule_cache_holds():
+    # T_q * G = 2048 rows make gangs of eight CTAs, i.e. 18 ranges of equal cost on 148 SMs.  With 64
+    # queries and probes (1, 2, 3, k) the 64 long pairs carry 17/18 of the cost, so the last range holds
+    # all 192 short pairs: far more than a CTA copies to shared memory, the rest of the schedule is read
+    # from the workspace.  Rows of short and long pairs are compared with the oracle.
+    ab = hp.gpu_binding()
+    B, k, probes, t_q = 64, 720, (1, 2, 3, 720), 128
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=1024, len_dist="const", len_lo=64, len_hi=64, batch=B, k=k, probes=probes,
+                                  t_q=t_q, n_q_heads=16, n_kv_heads=1, head_dim=64, seed=27)
+    pool = wl.make_pool(w, n_layers=1)
+    qs = wl.make_queries(w, n_layers=1)
+    rng = np.random.default_rng(5)
+    sel4 = np.stack([rng.permutation(1024)[:k] for _ in range(4)]).astype(np.int32)   # four selections, dealt out
+    ctx4 = _oracle_ctx(w, pool, sel4, 1)
+    L = k * 64
+    cap = L + 64
+    kc = torch.zeros((B, 1, cap, 1, 64), dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    off = torch.zeros((B, k + 1), dtype=torch.int64)
+    for b in range(B):
+        ok, ov, o = ctx4[b % 4]
+        kc[b, :, :L], vc[b, :, :L] = ok, ov
+        off[b] = torch.from_numpy(o)
+    model = hp.model_of(ab, w, n_layers=1)
+    out, lse, st = hp.run_attn(ab, model, kc.cuda(), vc.cuda(), cap, off.cuda(), k, list(probes),
+                               qs["q"].cuda(), qs["kq"].cuda(), qs["vq"].cuda(), 0, 1)
+    assert st == 0
+    out, lse = out.cpu(), lse.cpu()
+    got, want, rows = [], [], []
+    for j in range(len(probes)):
+        n_rows = 40 if j < 3 else 8                      # the short pairs are the ones behind the cache
+        for _ in range(n_rows):
+            rows.append((int(rng.integers(B)), j, int(rng.integers(t_q)), int(rng.integers(16))))
+    rows += [(63, 0, 127, 15), (0, 2, 0, 0), (63, 2, 127, 15)]        # the last pair of the call, and corners
+    for b, j, t, h in rows:
+        o_want, l_want = orc.attn_row(hp.f64(qs["q"][b, 0, j, t, h]), hp.f64(qs["kq"][b, 0, j]),
+                                      hp.f64(qs["vq"][b, 0, j]), hp.f64(kc[b, 0]), hp.f64(vc[b, 0]),
+                                      int(off[b, probes[j]]), t, 0, w.rope_base)
+        got.append(out[b, 0, j, t, h].double().numpy())
+        want.append(o_want)
+        assert abs(float(lse[b, 0, j, h, t]) - l_want) <= hp.lse_bound()
+    hp.assert_attn_close(np.stack(got), np.stack(want))

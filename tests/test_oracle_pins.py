@@ -317,6 +317,26 @@ def test_topk_ties_self_match_and_prefix_property():
         assert np.array_equal(orc.select_topk(qe, emb, n)[0][0], sel[0, :n])
 
 
+def test_min_adjacent_gap_on_hand_made_scores():
+    # q = e_x and shot i = (s_i, sqrt(1 - s_i^2)) give cosine s_i: the sorted scores and their gaps are known
+    s = np.array([0.10, 0.90, 0.50, 0.50, 0.49, 0.30, -0.20])
+    emb = np.stack([s, np.sqrt(1.0 - s * s)], axis=1) * np.array([1.0, 3.0, 0.5, 2.0, 1.0, 7.0, 1.0])[:, None]
+    qe = np.array([[2.0, 0.0]])
+    # ranks 1..4 are 0.9, 0.5, 0.5, 0.49: the true tie is skipped, the smallest real gap is 0.01
+    assert abs(orc.min_adjacent_gap(qe, emb, 3) - 0.01) < 1e-12
+    assert abs(orc.min_adjacent_gap(qe, emb, 1) - 0.40) < 1e-12          # 0.9 | 0.5
+    # the gap between rank k and rank k+1 counts (it decides who is selected): 0.49 | 0.30 is not reached at k = 3
+    assert abs(orc.min_adjacent_gap(qe, emb, 5) - 0.01) < 1e-12
+    assert abs(orc.min_adjacent_gap(qe, emb[[1, 5, 0]], 2) - 0.20) < 1e-12   # 0.9, 0.3, 0.1
+    # several queries: the smallest over the batch
+    q2 = np.array([[2.0, 0.0], [0.0, 1.0]])      # second query: cosines sqrt(1 - s^2)
+    c2 = np.sort(np.sqrt(1.0 - emb[[1, 5, 0], 0] ** 2 / (emb[[1, 5, 0]] ** 2).sum(1)))[::-1]
+    want = min(0.20, float(np.min(c2[:-1] - c2[1:])))
+    assert abs(orc.min_adjacent_gap(q2, emb[[1, 5, 0]], 2) - want) < 1e-12
+    # only exact ties (identical rows): nothing to report
+    assert orc.min_adjacent_gap(qe, np.array([[1.0, 1.0], [1.0, 1.0], [1.0, 1.0]]), 2) == np.inf
+
+
 # --------------------------------------------------------------- entropy
 def test_entropy_closed_forms_and_scipy():
     V = 1024
@@ -418,7 +438,7 @@ PIN_TESTS = [
     test_attention_probe_equals_standalone_call_and_prefix_only,
     test_attention_closed_forms, test_attention_scale_is_inverse_sqrt_head_dim,
     test_gqa_head_mapping, test_cosine_against_scipy_and_python_sort,
-    test_topk_ties_self_match_and_prefix_property,
+    test_topk_ties_self_match_and_prefix_property, test_min_adjacent_gap_on_hand_made_scores,
     test_entropy_closed_forms_and_scipy, test_threshold_rule_on_the_papers_case_study,
     test_subset_entropy_closed_forms_and_bounds, test_probe_rounds_on_the_papers_case_study,
 ]
@@ -486,6 +506,20 @@ def _mut_cosine_no_norm(q_emb, emb):
     return np.asarray(q_emb, dtype=np.float64) @ np.asarray(emb, dtype=np.float64).T
 
 
+def _mut_gap_always_inf(q_emb, emb, k):
+    return np.inf
+
+
+def _mut_gap_counts_ties(q_emb, emb, k):
+    s = _ORIG["cosine_scores"](q_emb, emb)
+    top = -np.sort(-s, axis=1)[:, : k + 1]
+    return float((top[:, :-1] - top[:, 1:]).min())              # a true tie gives 0
+
+
+def _mut_gap_stops_at_rank_k(q_emb, emb, k):
+    return _ORIG["min_adjacent_gap"](q_emb, emb, k - 1) if k > 1 else np.inf
+
+
 def _mut_first_ok_strict(H, tau, P):
     Hm = np.asarray(H).reshape(-1, P)
     return np.array([next((j for j in range(P) if Hm[b, j] > tau), -1)
@@ -545,6 +579,9 @@ _ORIG = {}
     ("entropy_subset", _mut_subset_always_renorm),
     ("entropy_subset", _mut_subset_local_softmax),
     ("cosine_scores", _mut_cosine_no_norm),
+    ("min_adjacent_gap", _mut_gap_always_inf),
+    ("min_adjacent_gap", _mut_gap_counts_ties),
+    ("min_adjacent_gap", _mut_gap_stops_at_rank_k),
     ("first_ok", _mut_first_ok_strict),
     ("probe_rounds", _mut_probe_rounds_lowest_entropy),
     ("probe_rounds", _mut_probe_rounds_runs_every_round),
@@ -555,7 +592,8 @@ _ORIG = {}
     ("attn_row", _mut_attn_row_factory("prefix")),
 ])
 def test_planted_mistakes_are_caught(name, mutant, monkeypatch):
-    for n in ("rope", "plan_offsets", "entropy", "entropy_subset", "probe_rounds"):
+    for n in ("rope", "plan_offsets", "entropy", "entropy_subset", "probe_rounds", "cosine_scores",
+              "min_adjacent_gap"):
         _ORIG[n] = getattr(orc, n)
     assert not _caught(), "pins must pass on the unmodified oracle"
     monkeypatch.setattr(orc, name, mutant)
