@@ -102,13 +102,41 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def resolve_workload(name: str, n_layers: int = 0) -> wl.Workload:
+HEADLINE = "cfg5"            # the largest 8B-shape configuration that fits one GPU
+SUB_WORKLOADS = ("cfg2", "cfg3")   # reported beside it in the default run, each with its own roofline / clocks / e2e
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/ (file named beside each figure).  A capture of a few layers / queries is scaled to a full
+# launch by the units it holds: (query, layer, kv head) units are independent and equally sized on
+# average, so the traffic grows in proportion.  None = no capture of the kernel as it stands.
+NCU_TRAFFIC = {
+    # workload: (attn_main bytes per captured launch, layers x queries in that capture,
+    #            gather bytes per captured launch, layers x queries in that capture)
+}
+
+
+def resolve_workload(name: str, n_layers: int = 0, n_queries: int = 0) -> wl.Workload:
     w = wl.CONFIGS[name]
     if n_layers:          # a stated smaller case of the same shape (profiling captures)
         w = w.scaled(n_layers=min(w.n_layers, n_layers))
-    if w.k == 0:      # cfg4: k = longest similarity-ordered prefix within the token limit; fixed at set-up
-        raise SystemExit("cfg4 is a parity configuration; bench workloads: cfg2 cfg3 cfg5")
+    if n_queries:
+        w = w.scaled(batch=min(w.batch, n_queries))
     return w
+
+
+def resolve_k_by_budget(ab, dpool, q_emb, w: wl.Workload, lengths: np.ndarray) -> wl.Workload:
+    """cfg4 names a token budget, not a shot count: k = the longest similarity-ordered prefix whose
+    total length stays within the budget (query 0 decides; fixed at set-up, outside the timed region)."""
+    dev = q_emb.device
+    n = int(dpool.c.n_shots)
+    sel = torch.empty((w.batch, n), dtype=torch.int32, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(max(256, ab.adapshot_select_workspace_bytes(n, w.batch, n)), dtype=torch.uint8, device=dev)
+    ab.adapshot_select(dpool, q_emb, n, sel, None, ws, st)
+    torch.cuda.synchronize()
+    order = sel[0].cpu().numpy()
+    k = int(np.searchsorted(np.cumsum(lengths[order]), w.ctx_token_limit, side="right"))
+    return w.scaled(k=k, probes=(k,))
 
 
 def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e9) -> int:
@@ -162,9 +190,10 @@ def oracle_sample_seconds(w: wl.Workload, pool, qs, row_stride: int):
     """Times the oracle, as it stands, on a bounded sample of the workload: select,
     offsets, assemble and entropy in full for query 0 / layer 0, attention on every
     `row_stride`-th (probe, head, token) row; returns (seconds scaled to one full step,
-    description, measured seconds)."""
+    description, measured seconds, CPU seconds used per second of wall clock)."""
     from oracle import adapshot_oracle as orc
     f64 = wl.to_f64
+    cpu0 = time.process_time()
     t0 = time.perf_counter()
     sel, _ = orc.select_topk(f64(qs["q_emb"]), f64(pool["emb"]), w.k)
     off = orc.plan_offsets(sel, pool["shot_off"])
@@ -183,11 +212,13 @@ def oracle_sample_seconds(w: wl.Workload, pool, qs, row_stride: int):
     orc.entropy(f64(qs["logits"]))
     t_entropy = time.perf_counter() - t0
     units = w.batch * w.n_layers                                   # (query, layer) units are independent
-    full = t_select + t_entropy + units * (t_assemble + t_attn * len(rows) / len(sample))
+    full = w.batch * (t_select + t_entropy) + units * (t_assemble + t_attn * len(rows) / len(sample))
     measured = t_select + t_assemble + t_attn + t_entropy
-    desc = (f"select+entropy full; assemble and attention for query 0, layer 0 with every {row_stride}th of "
-            f"{len(rows)} attention rows; scaled by rows and by {units} (query, layer) units")
-    return full, desc, measured, float(off[:, -1].sum())
+    desc = (f"query 0: select and entropy in full (scaled by {w.batch} queries), assemble and attention at layer 0 "
+            f"with every {row_stride}th of {len(rows)} attention rows (scaled by rows and by {units} (query, layer) "
+            "units)")
+    cores_used = (time.process_time() - cpu0) / max(measured, 1e-9)      # CPU seconds per second of wall clock
+    return full, desc, measured, cores_used
 
 
 def job_aggregate(ms: float, tokens: float, dist, device):
@@ -207,77 +238,146 @@ def rank_seed(seed: int, rank: int) -> int:
     return seed + 100 * rank if rank else seed
 
 
-def cpu_threads() -> int:
+def cpu_threads() -> dict:
+    """Threads the oracle run can use: its per-row loops are single-threaded Python, the numpy
+    products inside them go through the BLAS pool."""
+    blas = 1
     try:
         import threadpoolctl
         info = threadpoolctl.threadpool_info()
-        return max([i.get("num_threads", 1) for i in info] + [1])
+        blas = max([i.get("num_threads", 1) for i in info] + [1])
     except Exception:
-        return 1
+        pass
+    return {"python_threads": 1, "blas_threads": blas, "host_cores": os.cpu_count() or 1}
 
 
 def host_inputs(w: wl.Workload, n_pool_layers: int = 1):
-    """CPU copies of a one-layer slice of the workload for the oracle legs."""
+    """CPU copies of a one-layer, one-query slice of the workload for the oracle legs, and the
+    oracle's own selection / plan for the whole batch (cheap: one B x N x E product)."""
+    from oracle import adapshot_oracle as orc
     ws = w.scaled(batch=1)
     pool = wl.make_pool(ws, "cpu", n_layers=n_pool_layers)
+    q_emb_all = wl.make_query_embeddings(w, "cpu")
+    if w.k == 0:          # token-budget selection: the longest similarity-ordered prefix within the limit
+        order, _ = orc.select_topk(wl.to_f64(q_emb_all), wl.to_f64(pool["emb"]), int(pool["n_shots"]))
+        k = int(np.searchsorted(np.cumsum(pool["lengths"][order[0]]), w.ctx_token_limit, side="right"))
+        w = w.scaled(k=k, probes=(k,))
+        ws = w.scaled(batch=1)
     qs = wl.make_queries(ws, "cpu", n_layers=1)
-    return pool, qs
+    sel_all, _ = orc.select_topk(wl.to_f64(q_emb_all), wl.to_f64(pool["emb"]), w.k)
+    ctx_tokens = float(orc.plan_offsets(sel_all, pool["shot_off"])[:, -1].sum())
+    return w, pool, qs, ctx_tokens
+
+
+def workload_config(w: wl.Workload, pool_shots: int, pool_tokens: int, ctx_tokens: float, world: int) -> dict:
+    """The keys that name the workload: the same in the GPU arm's line and in the reference arm's."""
+    return {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
+            "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool_shots),
+            "pool_tokens": int(pool_tokens), "ctx_tokens_per_step": float(ctx_tokens),
+            "parallelism": "replicas" if world > 1 else "single"}      # (the selection is device-independent)
 
 
 def run_reference(args, w: wl.Workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    pool, qs = host_inputs(w)
+    w, pool, qs, ctx_tokens = host_inputs(w)
     n_rows = len(w.probes) * w.n_q_heads * w.t_q
     stride = max(1, n_rows // 96)
     for _ in range(args.warmup):
         oracle_sample_seconds(w, pool, qs, stride * 8)
-    vals, desc, meas, ctx_tokens = [], "", 0.0, 0.0
+    vals, desc, used = [], "", []
     for _ in range(args.steps):
-        full, desc, m, ctx1 = oracle_sample_seconds(w, pool, qs, stride)
+        full, desc, _m, c = oracle_sample_seconds(w, pool, qs, stride)
         vals.append(full)
-        meas += m
-        ctx_tokens = ctx1 * w.batch
+        used.append(c)
     sec = float(np.mean(vals))
     value = ctx_tokens / sec
+    cfg = workload_config(w, pool["n_shots"], pool["pool_tokens"], ctx_tokens, 1)
+    cfg["note"] = "oracle timed on host cores; each step is a bounded sample scaled to the full step"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "note": "oracle timed on host cores; each step is a bounded sample "
-                       "scaled to the full step"},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                             "sample": desc},
+            "config": cfg,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": max(1, round(float(np.mean(used)))),
+                             "cpu_seconds_per_second": float(np.mean(used)), "threads": cpu_threads(),
+                             "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------- GPU arm
-def run_ours(args, w: wl.Workload):
+def _timed(fn, n, flush):
+    """Mean device time of fn() over n calls, L2 flushed before each (CUDA events on the current stream)."""
+    tot = 0.0
+    for _ in range(n):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        tot += a.elapsed_time(b)
+    return tot / n
+
+
+def per_probe_costs(ab, path, model, dpool, w, qc, kqc, vqc, ctx_off_np, flush, n_rep=5):
+    """What every nested probe costs on its own, on the first layer chunk: the attention of that probe
+    alone over its prefix of the shared re-encoded cache, and the gather of the shots it adds to the
+    previous probe's prefix (the prefix itself is shared and stays in place)."""
+    lb, le = path.chunks[0]
+    nl = le - lb
+    k_ctx, v_ctx = path.ctx_views(nl)
+    out = []
+    dev = path.status.device
+    prev = 0
+    for j, n_j in enumerate(w.probes):
+        q_j, kq_j, vq_j = (x[0][:, :, j:j + 1].contiguous() for x in (qc, kqc, vqc))
+        o_j = torch.empty_like(q_j)
+        attn_ms = _timed(lambda: ab.adapshot_query_attn(model, k_ctx, v_ctx, path.ctx_cap, path.ctx_off, path.k,
+                                                        [n_j], q_j, kq_j, vq_j, lb, le, o_j, None, path.ws_attn,
+                                                        path.status), n_rep, flush)
+        sel_j = path.sel_idx[:, :n_j].contiguous()
+        off_j = torch.empty((w.batch, n_j + 1), dtype=torch.int64, device=dev)
+        gather_ms = _timed(lambda: ab.adapshot_assemble_kv_from(model, dpool, sel_j, prev, lb, le, k_ctx, v_ctx,
+                                                                path.ctx_cap, off_j, path.status), n_rep, flush)
+        Lj = ctx_off_np[:, n_j].astype(np.float64)
+        Lp = ctx_off_np[:, prev].astype(np.float64) if prev else np.zeros_like(Lj)
+        flops = float((4.0 * w.t_q * (Lj + (w.t_q + 1) / 2.0) * w.n_q_heads * w.head_dim).sum()) * nl
+        out.append({"n_shots": int(n_j), "ctx_tokens": float(Lj.sum()),
+                    "attn_ms": attn_ms * w.n_layers / nl, "attn_tflops": flops / (attn_ms * 1e-3) / 1e12,
+                    "gather_added_ms": gather_ms * w.n_layers / nl,
+                    "gather_added_gbs": float((Lj - Lp).sum()) * w.bytes_per_token_layer * 2 * nl
+                    / (gather_ms * 1e-3) / 1e9})
+        prev = n_j
+    path.assemble(lb, le, keep_plan=True)        # the cache of the whole selection again
+    torch.cuda.synchronize()
+    return {"what": "each nested probe alone (attention over its prefix; gather of the shots it adds), "
+                    f"measured on layers {lb}..{le - 1} and scaled to {w.n_layers} layers",
+            "probes": out,
+            "sum_attn_ms": float(sum(p["attn_ms"] for p in out)),
+            "sum_gather_ms": float(sum(p["gather_added_ms"] for p in out))}
+
+
+def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: int, world: int,
+            with_cpu_baseline: bool) -> dict:
+    """Builds one workload on the device, times the whole path over it and returns the fields of a
+    bench line for it (everything is freed again on return)."""
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    w = resolve_workload(name, args.layers, args.queries)
     if w.dtype != "bf16":   # cfg1: fp32 storage; the attention kernel takes bf16 (the parity tests round its inputs)
-        raise SystemExit(f"{w.name} is a parity configuration (fp32 storage); bench workloads: cfg2 cfg3 cfg5")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    peaks = load_peaks()
-    dev = torch.device("cuda", local)
+        raise SystemExit(f"{w.name} is a parity configuration (fp32 storage); bench workloads: cfg2 cfg3 cfg4 cfg5")
 
     # ---- resident inputs (every rank: same pool, its own queries)
     pool = wl.make_pool(w, dev)
-    wq = w.scaled(seed=rank_seed(w.seed, rank))
     so = torch.from_numpy(pool["shot_off"]).to(dev)
-    k_pool, v_pool = pool["k"], pool["v"]
-    dpool = ab.Pool(so, k_pool, v_pool, pool["emb"])
+    dpool = ab.Pool(so, pool["k"], pool["v"], pool["emb"])
+    wq = w.scaled(seed=rank_seed(w.seed, rank))
+    if w.k == 0:
+        w = resolve_k_by_budget(ab, dpool, wl.make_query_embeddings(wq, dev), w, pool["lengths"])
+        wq = w.scaled(seed=wq.seed)
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base,
                           k_pos_mode=args.k_pos_mode)
     qs = wl.make_queries(wq, dev)
@@ -286,7 +386,8 @@ def run_ours(args, w: wl.Workload):
     fused = args.variant == "fused"
     if fused and not args.layers_per_call:
         lpc = w.n_layers                      # no assembled cache to fit: all layers in one call
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused)
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused,
+                     entropy_overlap=args.entropy_overlap)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
     del qs
@@ -312,21 +413,25 @@ def run_ours(args, w: wl.Workload):
             dist.barrier()
         torch.cuda.synchronize()
 
+    def check_status(when):
+        code = int(path.status.item())
+        if code != 0:
+            raise SystemExit(f"device status {code} {when}: {ab.adapshot_strerror(code)}")
+
     step()
     torch.cuda.synchronize()
-    if path.status.item() != 0:
-        raise SystemExit(f"device status {path.status.item()}: {ab.adapshot_strerror(path.status.item())}")
+    check_status("after the first pass")
     ctx_off = path.ctx_off.cpu().numpy()
     counts = algorithmic_counts(w, ctx_off, w.n_layers)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         flush.zero_()
         step()
     barrier()
 
     # ---- timed region: K steps, CUDA events around every step, L2 flushed between steps
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    with ClockSampler(local) as clocks:
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    with ClockSampler(dev.index) as clocks:
         barrier()
         for a, b in ev:
             flush.zero_()
@@ -337,15 +442,14 @@ def run_ours(args, w: wl.Workload):
     step_ms = np.array([a.elapsed_time(b) for a, b in ev])
     total_ms = float(step_ms.sum())
     total_ms, job_tokens = job_aggregate(total_ms, counts["ctx_tokens"], dist, dev)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     value = job_tokens / (ms_per_step * 1e-3)
-    if path.status.item() != 0:
-        raise SystemExit(f"device status {path.status.item()} after the timed region")
+    check_status("after the timed region")
 
     # ---- per-call device times (second pass, same conditions) for the roofline object
     names = ["select", "assemble", "attn", "entropy"]     # select includes the plan; assemble = gather
     acc = {n: 0.0 for n in names}
-    n_prof = min(args.steps, 50)
+    n_prof = min(steps, 50)
     for _ in range(n_prof):
         flush.zero_()
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(2 + 2 * len(path.chunks) + 1)]
@@ -395,17 +499,21 @@ def run_ours(args, w: wl.Workload):
     n_main = len(path.chunks)
 
     attn_s = main_ms * 1e-3
+    call_s = per_call_ms["attn"] * 1e-3
     gather_s = per_call_ms["assemble"] * 1e-3
     attn_tflops = counts["attn_flops"] / attn_s / 1e12
     attn_kv_gbs = counts["attn_kv_bytes"] / attn_s / 1e9
     tensor_bound = counts["attn_flops"] / (peaks["bf16_tflops"] * 1e12) >= \
         counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
-    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in
-    # profiles/ (cfg3: a 2-layer capture scaled by the layers one launch processes)
-    traffic_attn = {"cfg2": 104.3e6, "cfg3": 2.2407e9 / 2 * path.lpc}.get(w.name) if not fused else None
-    traffic_gather = {"cfg2": 123.5e6, "cfg3": 4.2670e9 / 2 * path.lpc}.get(w.name)
-    if args.layers:
-        traffic_attn = traffic_gather = None
+    traffic_attn = traffic_gather = None
+    cap = NCU_TRAFFIC.get(w.name)
+    if cap is not None and not fused and not args.layers and not args.queries and args.k_pos_mode == 0:
+        units_per_launch = path.lpc * w.batch
+        if cap[0] is not None:
+            traffic_attn = cap[0] / cap[1] * units_per_launch
+        if cap[2] is not None:
+            traffic_gather = cap[2] / cap[3] * units_per_launch
+    call_tflops = counts["attn_flops"] / call_s / 1e12
     roofline = {
         "kernel": "attn_main_kernel" + ("<fused>" if fused else ""),
         "launches_per_step": n_main,
@@ -421,7 +529,7 @@ def run_ours(args, w: wl.Workload):
         "algorithmic_flops_per_launch": counts["attn_flops"] / n_main,
         "algorithmic_kv_bytes_per_launch": counts["attn_kv_bytes"] / n_main,
         "whole_call": {"what": "adapshot_query_attn (prep + main + combine)", "ms_per_step": per_call_ms["attn"],
-                       "achieved": counts["attn_flops"] / (per_call_ms["attn"] * 1e-3) / 1e12, "unit": "TFLOP/s"},
+                       "achieved": call_tflops, "unit": "TFLOP/s", "frac": call_tflops / peaks["bf16_tflops"]},
         "gather": None if fused else {
             "bound": "hbm", "achieved": counts["gather_bytes"] / gather_s / 1e9, "peak": peaks["hbm_gbs"],
             "unit": "GB/s", "frac": counts["gather_bytes"] / gather_s / 1e9 / peaks["hbm_gbs"],
@@ -431,6 +539,11 @@ def run_ours(args, w: wl.Workload):
         "entropy": {"bound": "hbm", "achieved": counts["entropy_bytes"] / (per_call_ms["entropy"] * 1e-3) / 1e9,
                     "unit": "GB/s", "ms_per_step": per_call_ms["entropy"]},
     }
+
+    per_probe = None
+    if len(w.probes) > 1 and not fused:
+        per_probe = per_probe_costs(ab, path, model, dpool, w, qc, kqc, vqc, ctx_off, flush)
+        check_status("after the per-probe pass")
 
     # ---- end to end: pinned host inputs in, results out, inside the timed region
     host = {"q_emb": q_emb.cpu().pin_memory(), "logits": logits.cpu().pin_memory(),
@@ -461,7 +574,7 @@ def run_ours(args, w: wl.Workload):
         else:
             path.run_host(host, dev_in, host_out, args.tau)
 
-    n_e2e = max(3, min(args.steps, 50))
+    n_e2e = max(3, min(steps, 50))
     for _ in range(3):
         e2e_step()
     barrier()
@@ -475,34 +588,142 @@ def run_ours(args, w: wl.Workload):
     e2e_ms = float(np.sum([a.elapsed_time(b) for a, b in ev2]))
     e2e_ms, _ = job_aggregate(e2e_ms, 0.0, dist, dev)
     e2e_value = job_tokens / (e2e_ms / n_e2e * 1e-3)
+    check_status("after the end-to-end pass")
+
+    config = workload_config(w, pool["n_shots"], pool["pool_tokens"], counts["ctx_tokens"], world)
+    config.update({"variant": args.variant, "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph,
+                   "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap,
+                   "entropy": "side stream, overlapped with the pass" if path.entropy_overlap
+                   else "after the last attention call (serial)",
+                   "l2": "flushed between steps (512 MiB write)"})
+    res = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": config, "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "graph": e2e_graph is not None},
+        "gpu_launches": launches_per_step * steps, "clocks": clocks.summary(),
+        "per_call_ms": per_call_ms,
+        "step_ms_min_med_max": [float(step_ms.min()), float(np.median(step_ms)), float(step_ms.max())],
+        "timed_region_ms": total_ms,
+    }
+    if per_probe is not None:
+        res["per_probe"] = per_probe
+
+    # ---- free everything this workload holds on the device and in pinned memory
+    del path, pool, dpool, so, qc, kqc, vqc, logits, q_emb, flush, host, out_host, dev_in, host_out, e2e_graph
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
 
     # ---- CPU oracle beside it (rank 0, N = 1 only)
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        hpool, hqs = host_inputs(w)
-        n_rows = len(w.probes) * w.n_q_heads * w.t_q
-        full, desc, meas, ctx1 = oracle_sample_seconds(w, hpool, hqs, max(1, n_rows // 3000))   # about 15 s of oracle work
-        cpu_baseline = {"value": ctx1 * w.batch / full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                        "sample": desc, "measured_seconds": meas}
+    if with_cpu_baseline:
+        w0, hpool, hqs, ctx_tokens = host_inputs(wl.CONFIGS[name] if not (args.layers or args.queries)
+                                                 else resolve_workload(name, args.layers, args.queries))
+        n_rows = len(w0.probes) * w0.n_q_heads * w0.t_q
+        full, desc, meas, used = oracle_sample_seconds(w0, hpool, hqs, max(1, n_rows // 3000))   # about 15 s of oracle work
+        res["cpu_baseline"] = {"value": ctx_tokens / full, "unit": UNIT, "cores": max(1, round(used)),
+                               "cpu_seconds_per_second": used, "threads": cpu_threads(),
+                               "kind": "oracle", "sample": desc, "measured_seconds": meas}
+    else:
+        res["cpu_baseline"] = None
+    return res
 
+
+def run_micro(args):
+    """One HBM-bound step alone on an input large enough to be bound by bandwidth (the benchmark
+    workloads give the entropy and selection steps a few MB, where they are bound by launch latency):
+    CUDA events around the call, L2 flushed before each, achieved GB/s against the measured copy peak.
+    Prints its own JSON line (not a bench line)."""
+    from paper_2605_03644_b200 import binding as ab
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    steps = args.steps or 20
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    if args.micro == "entropy":
+        R, V = args.rows, args.vocab
+        dt = torch.bfloat16 if args.logits_dtype == "bf16" else torch.float32
+        logits = torch.randn(R, V, generator=g, device=dev).to(dt)
+        H = torch.empty(R, dtype=torch.float32, device=dev)
+        fo = torch.empty(R, dtype=torch.int32, device=dev)
+        ws = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(R, V)), dtype=torch.uint8, device=dev)
+        fn = lambda: ab.adapshot_entropy(logits, H, args.tau, 1, fo, ws, st)
+        nbytes = float(R) * V * logits.element_size()
+        what = {"rows": R, "vocab": V, "logits_dtype": args.logits_dtype}
+    else:
+        w = wl.CONFIGS[HEADLINE if args.workload == "default" else args.workload]
+        n_shots = int(wl.shot_lengths(w).size)
+        emb = torch.randn(n_shots, w.emb_dim, generator=g, device=dev)
+        q_emb = torch.randn(w.batch, w.emb_dim, generator=g, device=dev)
+        so = torch.arange(n_shots + 1, dtype=torch.int64, device=dev)
+        dpool = ab.Pool(so, None, None, emb)
+        sel = torch.empty((w.batch, w.k), dtype=torch.int32, device=dev)
+        ws = torch.empty(max(256, ab.adapshot_select_workspace_bytes(n_shots, w.batch, w.k)), dtype=torch.uint8,
+                         device=dev)
+        fn = lambda: ab.adapshot_select(dpool, q_emb, w.k, sel, None, ws, st)
+        nbytes = float(n_shots) * w.emb_dim * 4
+        what = {"pool_shots": n_shots, "emb_dim": w.emb_dim, "queries": w.batch, "k": w.k}
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    with ClockSampler(dev.index) as clocks:
+        ms = _timed(fn, steps, flush)
+    if st.item() != 0:
+        raise SystemExit(f"device status {st.item()}")
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    print(json.dumps({"micro": args.micro, **what, "algorithmic_bytes": nbytes, "ms_per_call": ms, "steps": steps,
+                      "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                      "peak_source": f"of {peaks['source']}", "clocks": clocks.summary(),
+                      "l2": "flushed before every call (512 MiB write)"}))
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    dev = torch.device("cuda", local)
+    baseline = rank == 0 and world == 1 and not args.no_cpu_baseline
+
+    def steps_for(name, headline):
+        small = wl.CONFIGS[name].n_layers == 1 or args.layers == 1
+        if headline:
+            k = (2000 if small else 10) if args.steps is None else args.steps
+        else:       # a sub-workload's timed region lasts a few tenths of a second at least
+            k = max(2000 if small else 40, args.steps or 0)
+        wu = (20 if small else 3) if args.warmup is None else max(3, args.warmup)
+        return k, wu
+
+    if args.workload == "default":
+        free_bytes, _ = torch.cuda.mem_get_info()
+        headline = HEADLINE if free_bytes > 170e9 else "cfg3"      # cfg5 holds a 140 GB pool
+        subs = [n for n in SUB_WORKLOADS if n != headline]
+    else:
+        headline, subs = args.workload, []
+    sub_res = {}
+    for name in subs:
+        k, wu = steps_for(name, False)
+        sub_res[name] = measure(args, name, k, wu, dev, peaks, dist, rank, world, False)
+    k, wu = steps_for(headline, True)
+    line = measure(args, headline, k, wu, dev, peaks, dist, rank, world, baseline)
+    if sub_res:
+        line["workloads"] = sub_res
+        line["gpu_launches_all_workloads"] = line["gpu_launches"] + sum(r["gpu_launches"] for r in sub_res.values())
     if rank == 0:
-        clk = clocks.summary()
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "n_layers": w.n_layers, "batch_per_gpu": w.batch, "k": w.k,
-                       "probes": list(w.probes), "t_q": w.t_q, "pool_shots": int(pool["n_shots"]),
-                       "pool_tokens": int(pool["pool_tokens"]), "ctx_tokens_per_step": counts["ctx_tokens"],
-                       "variant": args.variant, "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph, "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap, "l2": "flushed between steps (512 MiB write)",
-                       "parallelism": "replicas" if world > 1 else "single"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "graph": e2e_graph is not None},
-            "gpu_launches": launches_per_step * args.steps, "clocks": clk,
-            "per_call_ms": per_call_ms,
-            "step_ms_min_med_max": [float(step_ms.min()), float(np.median(step_ms)), float(step_ms.max())],
-        }
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -514,9 +735,13 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="default",
+                    help="default: the headline configuration (cfg5) with cfg2 and cfg3 as sub-objects of the "
+                         "same line; or one of cfg2 cfg3 cfg4 cfg5 alone")
     ap.add_argument("--layers", type=int, default=0,
                     help="run only the first N layers of the workload (a smaller case for profiler captures)")
+    ap.add_argument("--queries", type=int, default=0,
+                    help="run only the first N queries of the workload (a smaller case for profiler captures)")
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
     ap.add_argument("--variant", default="materialise", choices=["materialise", "fused"],
@@ -527,19 +752,26 @@ def main():
                          "(the paper's store), the re-encode is one angle per shot")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the pass as one CUDA graph (auto: single-layer workloads)")
+    ap.add_argument("--entropy-overlap", action="store_true",
+                    help="run the entropy probe on a side stream beside the pass instead of after the attention")
+    ap.add_argument("--micro", default=None, choices=["entropy", "select"],
+                    help="time one HBM-bound step alone on a bandwidth-bound input and print its own JSON line")
+    ap.add_argument("--rows", type=int, default=2048, help="--micro entropy: logit rows")
+    ap.add_argument("--vocab", type=int, default=128256, help="--micro entropy: vocabulary size")
+    ap.add_argument("--logits-dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--tau", type=float, default=0.65)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    w = resolve_workload(args.workload, args.layers)
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
-        run_reference(args, w)
+        name = HEADLINE if args.workload == "default" else args.workload
+        run_reference(args, resolve_workload(name, args.layers, args.queries))
         return
-    small = w.n_layers == 1
-    args.steps = (1000 if small else 10) if args.steps is None else args.steps
-    args.warmup = (20 if small else 3) if args.warmup is None else max(3, args.warmup)
-    run_ours(args, w)
+    if args.micro is not None:
+        run_micro(args)
+        return
+    run_ours(args)
 
 
 if __name__ == "__main__":

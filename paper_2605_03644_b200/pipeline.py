@@ -22,7 +22,7 @@ from . import binding as ab
 class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
-                 overlap: bool = False, fused: bool = False, device="cuda"):
+                 overlap: bool = False, fused: bool = False, entropy_overlap: bool = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
@@ -51,8 +51,11 @@ class ReusePath:
         ws_fn = ab.adapshot_attn_fused_workspace_bytes if self.fused else ab.adapshot_attn_workspace_bytes
         self.ws_attn = torch.empty(max(256, ws_fn(model, batch, self.P, t_q, self.lpc, self.ctx_cap)), **u8)
         self.ws_entropy = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(batch * self.P, vocab)), **u8)
-        # the entropy probe depends on nothing else in the pass: it runs on a second stream
-        # (a parallel branch when the pass is captured into a graph)
+        # In the method the probe's logits come out of the model after the probe attention (Eq. 2
+        # follows Eq. 1), so the entropy step runs after the last attention call.  With
+        # entropy_overlap=True it runs on a second stream beside the pass instead (for callers
+        # whose logits are already there, e.g. those of the previous round of probes).
+        self.entropy_overlap = bool(entropy_overlap)
         self.side = torch.cuda.Stream(device=device)
         self.ev_begin, self.ev_entropy = torch.cuda.Event(), torch.cuda.Event()
         if self.overlap:
@@ -98,11 +101,12 @@ class ReusePath:
         gathers of a multi-chunk pass on the side stream, ordered by events).
         q_chunks[i] / kq_chunks[i] / vq_chunks[i] belong to layer chunk self.chunks[i]."""
         main = torch.cuda.current_stream()
-        self.ev_begin.record(main)
-        self.side.wait_event(self.ev_begin)
-        with torch.cuda.stream(self.side):
-            self.entropy(logits, tau)
-            self.ev_entropy.record(self.side)
+        if self.entropy_overlap:
+            self.ev_begin.record(main)
+            self.side.wait_event(self.ev_begin)
+            with torch.cuda.stream(self.side):
+                self.entropy(logits, tau)
+                self.ev_entropy.record(self.side)
         self.select(q_emb)
         if self.fused:
             self.plan()
@@ -127,7 +131,10 @@ class ReusePath:
                 main.wait_event(self.ev_asm[buf])
                 self.attend(q_chunks[i], kq_chunks[i], vq_chunks[i], self.out[i], lb, le, buf)
                 self.ev_attn[buf].record(main)
-        main.wait_event(self.ev_entropy)
+        if self.entropy_overlap:
+            main.wait_event(self.ev_entropy)
+        else:
+            self.entropy(logits, tau)
         return self.out, self.H, self.first_ok
 
     # ---- the same pass for a caller whose tensors live in host memory
@@ -138,8 +145,9 @@ class ReusePath:
         layer chunk), the same shapes on both sides; host_out: {"out": [...], "H", "first_ok",
         "sel_idx"}.  The query-side tensors go up on a copy stream while selection and the
         gather run, each chunk's output goes down on another while the next chunk is computed,
-        and the logits, the entropy and its results use the side stream: PCIe carries both
-        directions at once and the kernels wait only for the bytes they read.  Everything is
+        and the logits go up on the side stream (with entropy_overlap the entropy and its results
+        use it too): PCIe carries both directions at once and the kernels wait only for the bytes
+        they read.  Everything is
         joined back to the current stream before returning (the results are complete once that
         stream is synchronised), so the pass can also be captured into a graph."""
         if self.overlap:
@@ -156,9 +164,10 @@ class ReusePath:
             s.wait_event(self.ev_begin)
         with torch.cuda.stream(self.side):
             dev_in["logits"].copy_(host_in["logits"], non_blocking=True)
-            self.entropy(dev_in["logits"], tau)
-            host_out["H"].copy_(self.H, non_blocking=True)
-            host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
+            if self.entropy_overlap:
+                self.entropy(dev_in["logits"], tau)
+                host_out["H"].copy_(self.H, non_blocking=True)
+                host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
             self.ev_entropy.record(self.side)
         with torch.cuda.stream(self.h2d):
             for i in range(len(self.chunks)):
@@ -181,9 +190,13 @@ class ReusePath:
             with torch.cuda.stream(self.d2h):
                 self.d2h.wait_event(self.ev_out[i])
                 host_out["out"][i].copy_(self.out[i], non_blocking=True)
+        main.wait_event(self.ev_entropy)
+        if not self.entropy_overlap:          # the logits are up; the probe follows the last attention call
+            self.entropy(dev_in["logits"], tau)
+            host_out["H"].copy_(self.H, non_blocking=True)
+            host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
         self.ev_d2h.record(self.d2h)
         main.wait_event(self.ev_d2h)
-        main.wait_event(self.ev_entropy)
         return host_out
 
     # ---- the same pass as one CUDA graph: launch-bound small workloads (a few hundred

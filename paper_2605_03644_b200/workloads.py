@@ -125,9 +125,12 @@ def _gen(seed: int, device) -> torch.Generator:
     return g
 
 
-def _unit_rows(n: int, e: int, g: torch.Generator, device) -> torch.Tensor:
-    x = torch.randn(n, e, generator=g, device=device, dtype=torch.float32)
-    return x / x.norm(dim=1, keepdim=True)
+def _unit_rows(n: int, e: int, seed: int, device) -> torch.Tensor:
+    """Unit-norm Gaussian rows.  Always drawn by a CPU generator and then moved: the embeddings
+    decide the selection (and with it context lengths and token counts), which must not depend on
+    the device the large tensors are generated on."""
+    x = torch.randn(n, e, generator=_gen(seed, "cpu"), dtype=torch.float32)
+    return (x / x.norm(dim=1, keepdim=True)).to(device)
 
 
 def channel_scales(w: Workload, device, n_layers: Optional[int] = None):
@@ -160,9 +163,15 @@ def make_pool(w: Workload, device="cpu", n_layers: Optional[int] = None):
         x = torch.randn(tokens, w.n_kv_heads, w.head_dim, generator=g, device=device)
         v[l] = (x * sv[l]).to(w.torch_dtype)
         del x
-    emb = _unit_rows(len(lengths), w.emb_dim, g, device)
+    emb = _unit_rows(len(lengths), w.emb_dim, w.seed * 7919 + 13, device)
     return {"lengths": lengths, "shot_off": off, "k": k, "v": v, "emb": emb,
             "pool_tokens": tokens, "n_shots": len(lengths)}
+
+
+def make_query_embeddings(w: Workload, device="cpu") -> torch.Tensor:
+    """The q_emb of make_queries alone, for callers that need the selection of a whole batch
+    without the per-layer query tensors."""
+    return _unit_rows(w.batch, w.emb_dim, w.seed * 7919 + 29, device)
 
 
 def make_queries(w: Workload, device="cpu", n_layers: Optional[int] = None,
@@ -173,7 +182,7 @@ def make_queries(w: Workload, device="cpu", n_layers: Optional[int] = None,
     P = len(w.probes) if n_probes is None else n_probes
     g = _gen(w.seed * 7919 + 23, device)
     sk, sv = channel_scales(w, device, nl)
-    q_emb = _unit_rows(w.batch, w.emb_dim, g, device)
+    q_emb = make_query_embeddings(w, device)
     shape_q = (w.batch, nl, P, w.t_q, w.n_q_heads, w.head_dim)
     shape_kv = (w.batch, nl, P, w.t_q, w.n_kv_heads, w.head_dim)
     q = torch.randn(shape_q, generator=g, device=device).to(w.torch_dtype)
