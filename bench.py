@@ -384,17 +384,18 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
     lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap)
     fused = args.variant == "fused"
+    vpool = args.variant == "vpool"
     if fused and not args.layers_per_call:
         lpc = w.n_layers                      # no assembled cache to fit: all layers in one call
     path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused,
-                     entropy_overlap=args.entropy_overlap)
+                     entropy_overlap=args.entropy_overlap, vpool=vpool)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     q_emb, qc, kqc, vqc, logits = qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"]
     del qs
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     n_sel = 2 if w.n_shots <= 4096 else (3 if w.n_shots > 8192 else 2)
-    if fused:
-        launches_per_step = n_sel + 1 + len(path.chunks) * 4 + 2
+    if fused or vpool:
+        launches_per_step = n_sel + 1 + len(path.chunks) * ((1 if vpool else 0) + 4) + 2
     else:
         launches_per_step = n_sel + 1 + len(path.chunks) * (1 + 3) + 2
 
@@ -423,6 +424,8 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     check_status("after the first pass")
     ctx_off = path.ctx_off.cpu().numpy()
     counts = algorithmic_counts(w, ctx_off, w.n_layers)
+    if vpool:      # the gather moves K only: bpt / 2 read + bpt / 2 written per context token and layer
+        counts["gather_bytes"] *= 0.5
 
     for _ in range(warmup):
         flush.zero_()
@@ -507,7 +510,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
         counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
     traffic_attn = traffic_gather = None
     cap = NCU_TRAFFIC.get(w.name)
-    if cap is not None and not fused and not args.layers and not args.queries and args.k_pos_mode == 0:
+    if cap is not None and not fused and not vpool and not args.layers and not args.queries and args.k_pos_mode == 0:
         units_per_launch = path.lpc * w.batch
         if cap[0] is not None:
             traffic_attn = cap[0] / cap[1] * units_per_launch
@@ -541,7 +544,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     }
 
     per_probe = None
-    if len(w.probes) > 1 and not fused:
+    if len(w.probes) > 1 and not fused and not vpool:
         per_probe = per_probe_costs(ab, path, model, dpool, w, qc, kqc, vqc, ctx_off, flush)
         check_status("after the per-probe pass")
 
@@ -744,8 +747,9 @@ def main():
                     help="run only the first N queries of the workload (a smaller case for profiler captures)")
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
-    ap.add_argument("--variant", default="materialise", choices=["materialise", "fused"],
-                    help="materialise: gather + re-encode into a contiguous cache, then attend; "
+    ap.add_argument("--variant", default="materialise", choices=["materialise", "vpool", "fused"],
+                    help="materialise: gather + re-encode K and V into a contiguous cache, then attend; "
+                         "vpool: gather + re-encode K only, attention copies V tiles from the pool; "
                          "fused: attention reads the pool and re-encodes K in shared memory")
     ap.add_argument("--k-pos-mode", type=int, default=0, choices=[0, 1],
                     help="0: pool K carries no position (default); 1: pool K rotated at shot-local positions "

@@ -122,6 +122,10 @@ ADAPSHOT_API int adapshot_select(const adapshot_pool_t* pool, const float* q_emb
  *   the same sel_idx (an earlier call): it is then read, not written, so calls for
  *   further layer ranges may run on other streams while attention reads it.      */
 #define ADAPSHOT_ASSEMBLE_KEEP_PLAN 1u
+/*   ADAPSHOT_ASSEMBLE_K_ONLY: only k_ctx is written (v_ctx is ignored and may be NULL).  Eq. 7
+ *   corrects the keys alone, so a consumer that reads V from the pool through the plan
+ *   (adapshot_query_attn_vpool) needs no copy of it, and the gather moves half the bytes.    */
+#define ADAPSHOT_ASSEMBLE_K_ONLY 2u
 ADAPSHOT_API int adapshot_assemble_kv(const adapshot_model_t* model, const adapshot_pool_t* pool,
                          const int32_t* sel_idx, int32_t B, int32_t k,
                          int32_t layer_begin, int32_t layer_end,
@@ -192,6 +196,24 @@ ADAPSHOT_API size_t adapshot_attn_fused_workspace_bytes(const adapshot_model_t* 
 ADAPSHOT_API int adapshot_query_attn_fused(const adapshot_model_t* model, const adapshot_pool_t* pool,
                               const int32_t* sel_idx, const int64_t* ctx_off, int64_t ctx_cap,
                               int32_t B, int32_t k, const int32_t* probe_nshots, int32_t P,
+                              const void* q, const void* kq, const void* vq, int32_t Tq,
+                              int32_t layer_begin, int32_t layer_end, void* out, float* lse,
+                              uint32_t flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* ---- Step 3 over a cache that holds the re-encoded K only: the same attention, K tiles
+ * from k_ctx (written by adapshot_assemble_kv with ADAPSHOT_ASSEMBLE_K_ONLY), V tiles copied
+ * straight from the pool through sel_idx / ctx_off (Eq. 7 leaves V as it is, so its rows in
+ * the pool are the rows of the assembled context).  Results equal adapshot_query_attn over
+ * a full cache bit for bit in exact arithmetic (the same values reach the tensor cores; the
+ * accumulation order is the same).  ctx_cap: the capacity k_ctx was assembled with (it also
+ * sizes a row map of 2 * B * ctx_cap int32 in the workspace).  Needs pool_tokens < 2^31.
+ * Other arguments, limits and error rules as adapshot_query_attn.                        */
+ADAPSHOT_API size_t adapshot_attn_vpool_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
+                                           int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap);
+ADAPSHOT_API int adapshot_query_attn_vpool(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                              const int32_t* sel_idx, const void* k_ctx, int64_t ctx_cap,
+                              const int64_t* ctx_off, int32_t B, int32_t k,
+                              const int32_t* probe_nshots, int32_t P,
                               const void* q, const void* kq, const void* vq, int32_t Tq,
                               int32_t layer_begin, int32_t layer_end, void* out, float* lse,
                               uint32_t flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);

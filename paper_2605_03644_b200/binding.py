@@ -23,11 +23,13 @@ lib = C.CDLL(_LIB_PATH)
 OK, EINVAL, ESHAPE, EALIGN, ECAPACITY, EUNSUPPORTED, ECUDA, EINDEX, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7, -8
 F32, BF16 = 0, 1
 ASSEMBLE_KEEP_PLAN = 1
+ASSEMBLE_K_ONLY = 2
 
 EXPORTS = [
     "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv", "adapshot_assemble_kv_from",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
+    "adapshot_attn_vpool_workspace_bytes", "adapshot_query_attn_vpool",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_subset",
     "adapshot_entropy_static",
     "adapshot_profile", "adapshot_profile_attn_main_ms", "adapshot_selftest_wait_timeout",
@@ -81,6 +83,13 @@ _attn_fused_ws = _sig("adapshot_attn_fused_workspace_bytes", _sz,
                       [C.POINTER(ModelT), _i32, _i32, _i32, _i32, _i64])
 _attn_fused = _sig("adapshot_query_attn_fused", C.c_int,
                    [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _vp, _i64, _i32, _i32, C.POINTER(_i32), _i32,
+                    _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+
+
+_attn_vpool_ws = _sig("adapshot_attn_vpool_workspace_bytes", _sz,
+                      [C.POINTER(ModelT), _i32, _i32, _i32, _i32, _i64])
+_attn_vpool = _sig("adapshot_query_attn_vpool", C.c_int,
+                   [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _vp, _i64, _vp, _i32, _i32, C.POINTER(_i32), _i32,
                     _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
 
 
@@ -217,6 +226,25 @@ def adapshot_query_attn_fused(model: ModelT, pool: Pool, sel_idx: torch.Tensor, 
     arr = (_i32 * P)(*[int(x) for x in probe_nshots])
     _check(_attn_fused(C.byref(model), C.byref(pool.c), _ptr(sel_idx), _ptr(ctx_off), ctx_cap, B, k, arr, P,
                        _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
+                       flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_attn_vpool_workspace_bytes(model: ModelT, B: int, P: int, Tq: int, n_layers_in_call: int,
+                                        ctx_cap: int) -> int:
+    return _attn_vpool_ws(C.byref(model), B, P, Tq, n_layers_in_call, ctx_cap)
+
+
+def adapshot_query_attn_vpool(model: ModelT, pool: Pool, sel_idx: torch.Tensor, k_ctx: torch.Tensor,
+                              ctx_cap: int, ctx_off: torch.Tensor, probe_nshots: Sequence[int],
+                              q: torch.Tensor, kq: torch.Tensor, vq: torch.Tensor, layer_begin: int,
+                              layer_end: int, out: torch.Tensor, lse: Optional[torch.Tensor], ws: torch.Tensor,
+                              status: torch.Tensor, flags: int = 0):
+    B, k = sel_idx.shape
+    P = len(probe_nshots)
+    Tq = q.shape[3]
+    arr = (_i32 * P)(*[int(x) for x in probe_nshots])
+    _check(_attn_vpool(C.byref(model), C.byref(pool.c), _ptr(sel_idx), _ptr(k_ctx), ctx_cap, _ptr(ctx_off), B, k,
+                       arr, P, _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
                        flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
 
 

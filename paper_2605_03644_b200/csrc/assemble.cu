@@ -142,6 +142,7 @@ gather_rope_kernel(const GatherArgs a) {
   const uint4* vp = static_cast<const uint4*>(a.v_pool);
   uint4* kc = static_cast<uint4*>(a.k_ctx);
   uint4* vc = static_cast<uint4*>(a.v_ctx);
+  const bool with_v = vc != nullptr;               // a K-only cache: V is read from the pool by its consumer
 
   // A warp takes a run of kRun consecutive destination tokens of one query.  The plan lookup
   // (which selected shot covers the position) is a dependent chain of global loads, so it is
@@ -191,7 +192,7 @@ gather_rope_kernel(const GatherArgs a) {
           const long long dst = ((long long)b * a.n_layers_call + l) * layer_stride_ctx + p * row_vecs;
           for (int i = lane; i < row_vecs; i += 32) {
             kc[dst + i] = make_uint4(0, 0, 0, 0);
-            vc[dst + i] = make_uint4(0, 0, 0, 0);
+            if (with_v) vc[dst + i] = make_uint4(0, 0, 0, 0);
           }
         }
       }
@@ -253,7 +254,7 @@ gather_rope_kernel(const GatherArgs a) {
         }
       }
       // V: plain copy, four vectors in flight per lane
-      for (int i = lane; i < row_vecs; i += 128) {
+      for (int i = lane; with_v && i < row_vecs; i += 128) {
         uint4 r0 = vp[src + i];
         uint4 r1 = i + 32 < row_vecs ? vp[src + i + 32] : make_uint4(0, 0, 0, 0);
         uint4 r2 = i + 64 < row_vecs ? vp[src + i + 64] : make_uint4(0, 0, 0, 0);
@@ -308,18 +309,21 @@ extern "C" int adapshot_assemble_kv_from(const adapshot_model_t* model, const ad
                                          int32_t* status, void* stream) {
   if (model == nullptr || pool == nullptr || sel_idx == nullptr || ctx_off == nullptr) return ADAPSHOT_EINVAL;
   if (shot_begin < 0 || shot_begin >= k) return ADAPSHOT_ESHAPE;
-  if (B <= 0 || (flags & ~ADAPSHOT_ASSEMBLE_KEEP_PLAN) != 0 || pool->shot_off == nullptr || pool->n_shots <= 0)
+  if (B <= 0 || (flags & ~(ADAPSHOT_ASSEMBLE_KEEP_PLAN | ADAPSHOT_ASSEMBLE_K_ONLY)) != 0 ||
+      pool->shot_off == nullptr || pool->n_shots <= 0)
     return ADAPSHOT_EINVAL;
+  const bool k_only = (flags & ADAPSHOT_ASSEMBLE_K_ONLY) != 0;
+  if (k_only) v_ctx = nullptr;
   if (k < 1 || k > pool->n_shots) return ADAPSHOT_ESHAPE;
   const bool plan_only = k_ctx == nullptr && v_ctx == nullptr;
   const bool keep_plan = (flags & ADAPSHOT_ASSEMBLE_KEEP_PLAN) != 0;
   if (plan_only && keep_plan) return ADAPSHOT_EINVAL;
-  if (!plan_only && (k_ctx == nullptr || v_ctx == nullptr)) return ADAPSHOT_EINVAL;
+  if (!plan_only && (k_ctx == nullptr || (v_ctx == nullptr && !k_only))) return ADAPSHOT_EINVAL;
   if (((uintptr_t)sel_idx & 3u) || ((uintptr_t)ctx_off & 7u)) return ADAPSHOT_EALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   if (!plan_only) {
-    if (pool->k == nullptr || pool->v == nullptr) return ADAPSHOT_EINVAL;
+    if (pool->k == nullptr || (pool->v == nullptr && !k_only)) return ADAPSHOT_EINVAL;
     if (model->head_dim != 64 && model->head_dim != 128) return ADAPSHOT_ESHAPE;
     if (model->n_kv_heads <= 0 || model->n_q_heads % model->n_kv_heads != 0) return ADAPSHOT_ESHAPE;
     if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
@@ -327,7 +331,8 @@ extern "C" int adapshot_assemble_kv_from(const adapshot_model_t* model, const ad
     if (model->dtype != ADAPSHOT_F32 && model->dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
     if (model->k_pos_mode != 0 && model->k_pos_mode != 1) return ADAPSHOT_EUNSUPPORTED;
     if (!(model->rope_base > 1.0)) return ADAPSHOT_EINVAL;
-    if (!ads_aligned16(pool->k) || !ads_aligned16(pool->v) || !ads_aligned16(k_ctx) || !ads_aligned16(v_ctx))
+    if (!ads_aligned16(pool->k) || (!k_only && !ads_aligned16(pool->v)) || !ads_aligned16(k_ctx) ||
+        !ads_aligned16(v_ctx))
       return ADAPSHOT_EALIGN;
   }
 

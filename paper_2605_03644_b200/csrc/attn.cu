@@ -22,7 +22,10 @@
 // The fused variant (adapshot_query_attn_fused) adds attn_fused_plan (row map and rotary
 // table, once per call) and runs attn_main with two loader warps that copy the context
 // K/V tiles from the pool and re-encode K (Eq. 7) in shared memory, instead of TMA loads
-// from an assembled cache.
+// from an assembled cache.  The V-from-pool variant (adapshot_query_attn_vpool) sits between
+// the two: K tiles come by TMA from a cache that holds the re-encoded K only, V tiles (which
+// Eq. 7 leaves as they are) are copied from the pool through the row map, so that the gather
+// moves half the bytes.
 #include <cuda.h>
 #include <float.h>
 
@@ -41,7 +44,10 @@ constexpr int kUnitCost = 4;          // fixed cost of starting a unit, in tiles
 constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
 constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
-constexpr int kFusedThreads = 384;   // fused variant: warps 2-3 load and rotate K/V, softmax on warps 4-11
+constexpr int kFusedThreads = 384;   // fused / V-from-pool variants: warps 2-3 are loaders, softmax on warps 4-11
+constexpr int kModeCache = 0;        // K and V tiles by TMA from the assembled cache
+constexpr int kModeFused = 1;        // K and V tiles from the pool, K re-encoded in shared memory
+constexpr int kModeVPool = 2;        // K tiles by TMA from a K-only cache, V tiles from the pool
 constexpr int kLoaders = 64;         // threads of the two loader warps
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;   // log2 units: rescale O only when the max grows by 2^8
@@ -294,11 +300,11 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
 // The fused variant's loader warps take the stages of tile i+1 before they hand over tile i,
 // which needs a third V stage; the room goes at the expense of the read-out staging.
-template <int D, bool FUSED>
+template <int D, int MODE>
 struct AttnSmem {
   static constexpr int kKStages = 2;
-  static constexpr int kVStages = FUSED ? 3 : 2;
-  static constexpr uint32_t kStageBytes = FUSED ? 0 : 4096;               // per softmax warp: 32 rows x 128 bytes
+  static constexpr int kVStages = MODE == kModeFused ? 3 : 2;
+  static constexpr uint32_t kStageBytes = MODE == kModeFused ? 0 : 4096;  // per softmax warp: 32 rows x 128 bytes
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
   static constexpr uint32_t kOffQ = 0;                                    // Q of M tile A, then of M tile B
   static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
@@ -427,19 +433,21 @@ __device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, 
 // FUSED: the context K/V tiles are read from the pool through the row map (per-thread async
 // copies into the swizzled tile layout) and K is rotated in shared memory by two loader warps,
 // so that no re-encoded cache is ever written to HBM; TMA then only brings Q.
-template <int D, bool FUSED>
-__global__ void __launch_bounds__(FUSED ? kFusedThreads : kAttnThreads, 1)
+template <int D, int MODE>
+__global__ void __launch_bounds__(MODE != kModeCache ? kFusedThreads : kAttnThreads, 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
                  const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
-  using SM = AttnSmem<D, FUSED>;
+  constexpr bool FUSED = MODE == kModeFused;
+  constexpr bool VPOOL = MODE == kModeVPool;
+  using SM = AttnSmem<D, MODE>;
   constexpr int SUB = D / 64;
   constexpr int KS = SM::kKStages, VS = SM::kVStages;
   constexpr uint32_t kTileBytes = SM::kTileBytes;
   constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, 0);
   constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, 1);
   constexpr uint32_t kTmemS = 0, kTmemO = 256;
-  constexpr int kSoftmaxWarp0 = FUSED ? 4 : 2;          // first of the eight softmax warps
+  constexpr int kSoftmaxWarp0 = MODE != kModeCache ? 4 : 2;   // first of the eight softmax warps
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -467,7 +475,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int i = 0; i < 3; ++i) {
       mbar_init(bar(kBarKFull + i), FUSED ? kLoaders : 1);
       mbar_init(bar(kBarKEmpty + i), 1);
-      mbar_init(bar(kBarVFull + i), FUSED ? kLoaders : 1);
+      mbar_init(bar(kBarVFull + i), FUSED ? kLoaders : (VPOOL ? 32 : 1));
       mbar_init(bar(kBarVEmpty + i), 1);
     }
     mbar_init(bar(kBarDrain), 1);
@@ -548,15 +556,17 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               tma_load_4d(base + SM::kOffK + sk * kTileBytes + s * 16384u, mk, bar(kBarKFull + sk), s * 64, w.g, row,
                           outer);
             ++tk;
-            const int sv = tv % VS;
-            ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
+            if constexpr (!VPOOL) {
+              const int sv = tv % VS;
+              ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
+              if (!ok) break;
+              mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
 #pragma unroll
-            for (int s = 0; s < SUB; ++s)
-              tma_load_4d(base + SM::kOffV + sv * kTileBytes + s * 16384u, mv, bar(kBarVFull + sv), s * 64, w.g, row,
-                          outer);
-            ++tv;
+              for (int s = 0; s < SUB; ++s)
+                tma_load_4d(base + SM::kOffV + sv * kTileBytes + s * 16384u, mv, bar(kBarVFull + sv), s * 64, w.g,
+                            row, outer);
+              ++tv;
+            }
           }
         }
       }
@@ -564,8 +574,9 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // gave up: let the copies already in flight land before the CTA retires
         for (uint32_t t = tk > (uint32_t)KS ? tk - KS : 0; t < tk; ++t)
           mbar_wait(bar(kBarKFull + t % KS), (t / KS) & 1, abort_flag + 1);
-        for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
-          mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
+        if constexpr (!VPOOL)
+          for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
+            mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
       }
       if (!ok) {
         for (int x = 0; x < 2; ++x)
@@ -818,6 +829,64 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
     cp_async_wait<0>();
+  } else if (VPOOL && warp < 4) {
+    // --------------------------------------- loader: V tiles straight from the pool
+    // Eq. 7 corrects K only, so V needs no assembled copy: the tile's 128 context positions are
+    // looked up in the row map and their rows copied from the pool by per-thread async copies
+    // (zero fill beyond the context) into the swizzled layout the PV descriptors expect.  Warp 2
+    // serves the even tiles of the CTA's tile sequence, warp 3 the odd ones, each with one tile in
+    // flight; a lane copies the same 16-byte column of CPR-spaced rows, so a warp instruction
+    // reads whole 128- or 256-byte rows.
+    constexpr int CPR = D / 8;                 // 16-byte chunks per row
+    constexpr int RPI = 32 / CPR;              // rows per warp instruction
+    constexpr int NU = kTileN / RPI;           // copies per lane and tile
+    const uint32_t par = (uint32_t)(warp - 2);
+    const int c = lane % CPR, rsub = lane / CPR;
+    const uint32_t col_off = (uint32_t)(c / 8) * 16384u;
+    const int j = c & 7;
+    uint32_t tv = 0;
+    bool ok = true;
+    Walker wk = wk0;
+    Piece pc;
+    while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
+      for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
+        Item w;
+        make_item(p, pc, gang_id, mp, w);
+        for (int i = 0; i < w.n_tiles; ++i, ++tv) {
+          if ((tv & 1u) != par) continue;
+          const uint32_t sv = tv % VS;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag));
+          if (!ok) break;
+          const bool own = i >= w.n_ctx;
+          long long src_row[4];                 // source row (in rows of D elements) of tile rows lane + 32 q
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int row = lane + 32 * q4;
+            if (!own) {
+              const long long pos = (long long)(w.ctx_begin + i) * kTileN + row;
+              const int r = pos < p.ctx_cap ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
+              src_row[q4] = r < 0 ? -1 : ((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g;
+            } else {
+              const int t = (w.own_begin + i - w.n_ctx) * kTileN + row;
+              src_row[q4] = t >= p.Tq ? -1 : ((long long)w.outer_own * p.Tq + t) * p.Hkv + w.g;
+            }
+          }
+          const __nv_bfloat16* vb = own ? p.vq : p.v_pool;
+          const uint32_t v_base = base + SM::kOffV + sv * kTileBytes + col_off;
+#pragma unroll
+          for (int u = 0; u < NU; ++u) {
+            const int row = u * RPI + rsub;
+            const long long sr = __shfl_sync(0xffffffffu, src_row[(u * RPI) / 32], row & 31);
+            const __nv_bfloat16* g = vb + (sr < 0 ? 0 : sr) * D + c * 8;
+            cp_async16(v_base + row * 128u + ((uint32_t)(j ^ (row & 7)) << 4), g, sr < 0 ? 0u : 16u);
+          }
+          cp_async_commit();
+          cp_async_wait<0>();
+          fence_proxy_async_smem();
+          mbar_arrive(bar(kBarVFull + sv));
+        }
+      }
+    }
   } else {
     // ---------------------------------------------------- softmax + read-out of O
     const int x = (warp - kSoftmaxWarp0) >> 2;     // 0: M tile A, 1: M tile B
@@ -1186,7 +1255,8 @@ struct FusedSrc {
 
 // The gang (CTAs that walk the same K/V tiles, one M pair each per round) is the number of
 // M pairs when that is at most kMaxGang, else the M pairs are dealt out in rounds.
-AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, long long fused_ctx_cap = 0) {
+AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, long long fused_ctx_cap = 0,
+                   bool with_table = true) {
   AttnPlan pl;
   const int G = model->n_q_heads / model->n_kv_heads;
   const int D = model->head_dim;
@@ -1204,7 +1274,7 @@ AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, 
   pl.off_rowmap = pl.off_offmap = pl.off_tab = off;
   pl.tab_rows = 0;
   if (fused_ctx_cap > 0) {
-    pl.tab_rows = (fused_ctx_cap + kTileN - 1) / kTileN * kTileN;
+    pl.tab_rows = with_table ? (fused_ctx_cap + kTileN - 1) / kTileN * kTileN : 0;
     pl.off_rowmap = off; off += ads_round_up((size_t)B * fused_ctx_cap * 4, 256);
     pl.off_offmap = off; off += ads_round_up((size_t)B * fused_ctx_cap * 4, 256);
     pl.off_tab = off;    off += ads_round_up((size_t)pl.tab_rows * (D / 2) * 8, 256);
@@ -1222,7 +1292,8 @@ template <int D>
 int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx, int64_t ctx_cap,
                 const int64_t* ctx_off, int B, int k, const int32_t* probe_nshots, int P, const void* q,
                 const void* kq, const void* vq, int Tq, int nl, void* out, float* lse, const AttnPlan& pl,
-                void* ws, int32_t* status, cudaStream_t st, const FusedSrc* fused = nullptr) {
+                void* ws, int32_t* status, cudaStream_t st, const FusedSrc* fused = nullptr,
+                int mode = kModeCache) {
   const int Hq = model->n_q_heads, Hkv = model->n_kv_heads, G = Hq / Hkv;
   unsigned char* wsb = static_cast<unsigned char*>(ws);
   __nv_bfloat16* q_rot = reinterpret_cast<__nv_bfloat16*>(wsb + pl.off_qrot);
@@ -1248,13 +1319,10 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)ctx_cap, (uint64_t)B * nl};
     const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, (uint64_t)ctx_cap * Hkv * D * 2};
     const uint32_t box[4] = {64, 1, (uint32_t)kTileN, 1};
-    if (fused != nullptr) {
-      tm_kctx = tm_q;                  // never used: the loader warps read the pool
-      tm_vctx = tm_q;
-    } else {
-      if (!make_map(&tm_kctx, k_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
-      if (!make_map(&tm_vctx, v_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
-    }
+    tm_kctx = tm_q;                    // (a map the mode never uses: its loader warps read the pool)
+    tm_vctx = tm_q;
+    if (mode != kModeFused && !make_map(&tm_kctx, k_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    if (mode == kModeCache && !make_map(&tm_vctx, v_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
   }
   {
     const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)Tq, (uint64_t)B * nl * P};
@@ -1305,12 +1373,12 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   ap.n_mt = pl.n_mt; ap.n_mp = pl.n_mp; ap.gang = pl.gang; ap.n_gangs = n_gangs;
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
-  const int smem = (int)AttnSmem<128, false>::kTotal;     // same request for D = 64 and for the fused variant: one CTA per SM
-  static bool attr_done[2][kAdsMaxDevices] = {{false}, {false}};   // per template instance (D) and device
+  const int smem = (int)AttnSmem<128, kModeCache>::kTotal;     // same request for D = 64 and for the fused variant: one CTA per SM
+  static bool attr_done[3][kAdsMaxDevices] = {{false}, {false}, {false}};   // per template instance (D, mode) and device
   if (g_profile) ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[0], st));
-  if (fused == nullptr) {
-    if (ads_set_max_smem(attn_main_kernel<D, false>, smem, attr_done[0]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
-    attn_main_kernel<D, false><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(
+  if (mode == kModeCache) {
+    if (ads_set_max_smem(attn_main_kernel<D, kModeCache>, smem, attr_done[0]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+    attn_main_kernel<D, kModeCache><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(
         tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
   } else {
     ap.k_pool = static_cast<const __nv_bfloat16*>(fused->pool->k);
@@ -1320,9 +1388,15 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     ap.row_map = row_map; ap.off_map = off_map; ap.k_pos_mode = model->k_pos_mode; ap.rope_tab = rope_tab;
     ap.pool_tokens = fused->pool->pool_tokens; ap.ctx_cap = ctx_cap;
     ap.layer_begin = fused->layer_begin; ap.rope_base_f = model->rope_base;
-    if (ads_set_max_smem(attn_main_kernel<D, true>, smem, attr_done[1]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
-    attn_main_kernel<D, true><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
-        tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+    if (mode == kModeFused) {
+      if (ads_set_max_smem(attn_main_kernel<D, kModeFused>, smem, attr_done[1]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+      attn_main_kernel<D, kModeFused><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
+          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+    } else {
+      if (ads_set_max_smem(attn_main_kernel<D, kModeVPool>, smem, attr_done[2]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+      attn_main_kernel<D, kModeVPool><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
+          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+    }
   }
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
   if (g_profile) {
@@ -1427,9 +1501,55 @@ extern "C" int adapshot_query_attn_fused(const adapshot_model_t* model, const ad
   src.pool = pool; src.sel_idx = sel_idx; src.layer_begin = layer_begin;
   if (model->head_dim == 128)
     return launch_attn<128>(model, nullptr, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl,
-                            out, lse, pl, ws, status, st, &src);
+                            out, lse, pl, ws, status, st, &src, kModeFused);
   return launch_attn<64>(model, nullptr, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
-                         lse, pl, ws, status, st, &src);
+                         lse, pl, ws, status, st, &src, kModeFused);
+}
+
+extern "C" size_t adapshot_attn_vpool_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t P,
+                                                      int32_t Tq, int32_t n_layers_in_call, int64_t ctx_cap) {
+  if (model == nullptr || !attn_shape_ok(model) || B <= 0 || P <= 0 || Tq <= 0 || n_layers_in_call <= 0 ||
+      ctx_cap <= 0)
+    return 0;
+  return make_plan(model, B, P, Tq, n_layers_in_call, ctx_cap, false).total;
+}
+
+extern "C" int adapshot_query_attn_vpool(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                                         const int32_t* sel_idx, const void* k_ctx, int64_t ctx_cap,
+                                         const int64_t* ctx_off, int32_t B, int32_t k,
+                                         const int32_t* probe_nshots, int32_t P, const void* q, const void* kq,
+                                         const void* vq, int32_t Tq, int32_t layer_begin, int32_t layer_end,
+                                         void* out, float* lse, uint32_t flags, void* ws, size_t ws_bytes,
+                                         int32_t* status, void* stream) {
+  if (model == nullptr || pool == nullptr || sel_idx == nullptr || k_ctx == nullptr || ctx_off == nullptr ||
+      probe_nshots == nullptr || q == nullptr || kq == nullptr || vq == nullptr || out == nullptr || ws == nullptr)
+    return ADAPSHOT_EINVAL;
+  if (pool->v == nullptr || pool->shot_off == nullptr || pool->n_shots <= 0 || pool->pool_tokens <= 0)
+    return ADAPSHOT_EINVAL;
+  if (B <= 0 || k <= 0 || Tq <= 0 || ctx_cap <= 0 || flags != 0) return ADAPSHOT_EINVAL;
+  if (model->dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
+  if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
+  if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
+  if (P < 1 || P > kMaxProbes || (long long)P * B > kMaxPairs || k > pool->n_shots) return ADAPSHOT_ESHAPE;
+  for (int i = 0; i < P; ++i) {
+    if (probe_nshots[i] < 1 || probe_nshots[i] > k) return ADAPSHOT_ESHAPE;
+    if (i > 0 && probe_nshots[i] <= probe_nshots[i - 1]) return ADAPSHOT_ESHAPE;
+  }
+  if (!ads_aligned16(pool->v) || !ads_aligned16(k_ctx) || !ads_aligned16(q) || !ads_aligned16(kq) ||
+      !ads_aligned16(vq) || !ads_aligned16(out) || ((uintptr_t)ws & 255u) || ((uintptr_t)sel_idx & 3u))
+    return ADAPSHOT_EALIGN;
+  if (ctx_cap > (1ll << 31) - 256 || pool->pool_tokens > (1ll << 31) - 1) return ADAPSHOT_ESHAPE;
+  const int nl = layer_end - layer_begin;
+  const AttnPlan pl = make_plan(model, B, P, Tq, nl, ctx_cap, false);
+  if (ws_bytes < pl.total) return ADAPSHOT_ECAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FusedSrc src;
+  src.pool = pool; src.sel_idx = sel_idx; src.layer_begin = layer_begin;
+  if (model->head_dim == 128)
+    return launch_attn<128>(model, k_ctx, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out,
+                            lse, pl, ws, status, st, &src, kModeVPool);
+  return launch_attn<64>(model, k_ctx, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out, lse,
+                         pl, ws, status, st, &src, kModeVPool);
 }
 
 extern "C" int adapshot_profile(int enable) {

@@ -4,7 +4,8 @@ It owns the device buffers (assembled cache, offsets, workspaces, outputs) so a
 caller can run many queries without allocating; it does no arithmetic itself.
 Layers are processed in chunks of `layers_per_call`: assemble the chunk's cache,
 attend over it, reuse the buffer for the next chunk.  `fused=True` skips the assembled
-cache: attention reads the pool and re-encodes K on the fly.  `overlap=True` double-buffers the
+cache: attention reads the pool and re-encodes K on the fly.  `vpool=True` assembles the
+re-encoded K only and lets attention read V from the pool (the re-encode leaves V as it is).  `overlap=True` double-buffers the
 cache and enqueues the gather of chunk i+1 on a second stream; on B200 the persistent
 attention CTAs leave no room for a second resident kernel, so the two do not actually run
 together and the default is off.  Query-side tensors come as one tensor per chunk, [B][layers in chunk][P][T_q][heads][d] (in a model, the queries of a
@@ -22,7 +23,8 @@ from . import binding as ab
 class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
-                 overlap: bool = False, fused: bool = False, entropy_overlap: bool = False, device="cuda"):
+                 overlap: bool = False, fused: bool = False, entropy_overlap: bool = False,
+                 vpool: bool = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
@@ -38,17 +40,19 @@ class ReusePath:
         self.ctx_off = torch.empty((batch, k + 1), dtype=torch.int64, device=device)
         self.chunks = [(lb, min(self.nl, lb + self.lpc)) for lb in range(0, self.nl, self.lpc)]
         self.fused = bool(fused)
+        self.vpool = bool(vpool) and not self.fused
         self.overlap = bool(overlap) and len(self.chunks) > 1 and not self.fused
         n_ctx = batch * self.lpc * self.ctx_cap * hkv * d
         n_buf = 0 if self.fused else (2 if self.overlap else 1)     # the fused variant has no assembled cache
         self.k_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
-        self.v_bufs = [torch.empty(n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
+        self.v_bufs = [torch.empty(0 if self.vpool else n_ctx, dtype=dt, device=device) for _ in range(n_buf)]
         self.out = [torch.empty((batch, le - lb, self.P, t_q, hq, d), dtype=dt, device=device)
                     for lb, le in self.chunks]
         self.H = torch.empty((batch * self.P,), dtype=torch.float32, device=device)
         self.first_ok = torch.empty((batch,), dtype=torch.int32, device=device)
         self.ws_select = torch.empty(max(256, ab.adapshot_select_workspace_bytes(pool.c.n_shots, batch, k)), **u8)
-        ws_fn = ab.adapshot_attn_fused_workspace_bytes if self.fused else ab.adapshot_attn_workspace_bytes
+        ws_fn = (ab.adapshot_attn_fused_workspace_bytes if self.fused else
+                 ab.adapshot_attn_vpool_workspace_bytes if self.vpool else ab.adapshot_attn_workspace_bytes)
         self.ws_attn = torch.empty(max(256, ws_fn(model, batch, self.P, t_q, self.lpc, self.ctx_cap)), **u8)
         self.ws_entropy = torch.empty(max(256, ab.adapshot_entropy_workspace_bytes(batch * self.P, vocab)), **u8)
         # In the method the probe's logits come out of the model after the probe attention (Eq. 2
@@ -74,16 +78,21 @@ class ReusePath:
     def ctx_views(self, nl: int, buf: int = 0):
         shape = (self.B, nl, self.ctx_cap, self.model.n_kv_heads, self.model.head_dim)
         n = shape[0] * shape[1] * shape[2] * shape[3] * shape[4]
-        return self.k_bufs[buf][:n].view(shape), self.v_bufs[buf][:n].view(shape)
+        return self.k_bufs[buf][:n].view(shape), (None if self.vpool else self.v_bufs[buf][:n].view(shape))
 
     def assemble(self, layer_begin: int, layer_end: int, buf: int = 0, keep_plan: bool = False):
         k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin, buf)
+        flags = (ab.ASSEMBLE_KEEP_PLAN if keep_plan else 0) | (ab.ASSEMBLE_K_ONLY if self.vpool else 0)
         ab.adapshot_assemble_kv(self.model, self.pool, self.sel_idx, layer_begin, layer_end,
-                                k_ctx, v_ctx, self.ctx_cap, self.ctx_off, self.status,
-                                flags=ab.ASSEMBLE_KEEP_PLAN if keep_plan else 0)
+                                k_ctx, v_ctx, self.ctx_cap, self.ctx_off, self.status, flags=flags)
 
     def attend(self, q, kq, vq, out, layer_begin: int, layer_end: int, buf: int = 0):
         k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin, buf)
+        if self.vpool:
+            ab.adapshot_query_attn_vpool(self.model, self.pool, self.sel_idx, k_ctx, self.ctx_cap, self.ctx_off,
+                                         self.probes, q, kq, vq, layer_begin, layer_end, out, None,
+                                         self.ws_attn, self.status)
+            return
         ab.adapshot_query_attn(self.model, k_ctx, v_ctx, self.ctx_cap, self.ctx_off,
                                self.k, self.probes, q, kq, vq, layer_begin, layer_end, out, None,
                                self.ws_attn, self.status)

@@ -44,7 +44,7 @@ def _context_of(pool, sel_row, layer, g, L, base):
     return k_ctx[:, None, :], v_rows[:, None, :]      # [L, 1 head, d]
 
 
-def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=False):
+def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=False, vpool=False):
     from bench import layers_per_call_for
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
@@ -69,7 +69,7 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=Fa
     # ---- the CUDA path, as the benchmark launches it
     dpool = ab.Pool(torch.from_numpy(pool["shot_off"]).to(dev), pool["k"], pool["v"], pool["emb"])
     model = ab.make_model(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
-    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused)
+    path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused, vpool=vpool)
     chunk = lambda x: [x[:, lb:le].contiguous() for lb, le in path.chunks]
     tau = 0.65
     path.run(qs["q_emb"], chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]), qs["logits"], tau)
@@ -121,7 +121,8 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=Fa
         s, o = int(sel[b, r]), int(off[b, r])
         a0, a1 = int(so[s]), int(so[s + 1])
         T = a1 - a0
-        assert torch.equal(v_ctx_d[b, l - lb, o:o + T], pool["v"][l, a0:a1]), "V must be a bit copy"
+        if not vpool:        # (the V-from-pool variant keeps no copy of V)
+            assert torch.equal(v_ctx_d[b, l - lb, o:o + T], pool["v"][l, a0:a1]), "V must be a bit copy"
         want = torch.from_numpy(orc.rope(hp.f64(pool["k"][l, a0:a1]),
                                          (o + np.arange(T, dtype=np.float64))[:, None], w.rope_base))
         got_k = k_ctx_d[b, l - lb, o:o + T].cpu()
@@ -133,9 +134,11 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=Fa
     b, l = int(rng.integers(w.batch)), int(rng.integers(lb, le))
     L = int(off[b, -1])
     idx = np.concatenate([np.arange(so[s], so[s + 1]) for s in sel[b]])
-    assert torch.equal(v_ctx_d[b, l - lb, :L], pool["v"][l].index_select(0, torch.from_numpy(idx).to(dev)))
     pad_end = min(-(-L // 128) * 128, ctx_cap)
-    assert (k_ctx_d[b, l - lb, L:pad_end] == 0).all() and (v_ctx_d[b, l - lb, L:pad_end] == 0).all()
+    assert (k_ctx_d[b, l - lb, L:pad_end] == 0).all()
+    if not vpool:
+        assert torch.equal(v_ctx_d[b, l - lb, :L], pool["v"][l].index_select(0, torch.from_numpy(idx).to(dev)))
+        assert (v_ctx_d[b, l - lb, L:pad_end] == 0).all()
     del path, pool, qs, dpool, k_ctx_d, v_ctx_d
     gc.collect()
     torch.cuda.empty_cache()
@@ -163,3 +166,15 @@ def test_cfg2_full_size_fused_variant():
 
 def test_cfg3_full_size_fused_variant():
     _fullsize("cfg3", fused=True)
+
+
+def test_cfg2_full_size_v_from_pool_variant():
+    _fullsize("cfg2", n_combos=8, rows_per_combo=32, vpool=True)
+
+
+def test_cfg3_full_size_v_from_pool_variant():
+    _fullsize("cfg3", vpool=True)
+
+
+def test_cfg5_full_size_v_from_pool_variant():
+    _fullsize("cfg5", vpool=True)

@@ -27,13 +27,14 @@ def oracle_path(w, pool, qs, nl, tau, k_pos_mode=0):
     return sel, off, np.stack(outs), H, orc.first_ok(H, tau, len(w.probes))
 
 
-def run_gpu_path(w, pool, qs, nl, tau, layers_per_call=None, ctx_cap=None, overlap=False, fused=False):
+def run_gpu_path(w, pool, qs, nl, tau, layers_per_call=None, ctx_cap=None, overlap=False, fused=False, vpool=False):
     from paper_2605_03644_b200 import binding as ab
     from paper_2605_03644_b200.pipeline import ReusePath
     dp = hp.dev_pool(ab, pool)
     model = hp.model_of(ab, w, n_layers=nl)
     cap = ctx_cap or w.k * w.len_hi
-    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, cap, layers_per_call, overlap=overlap, fused=fused)
+    path = ReusePath(model, dp, w.batch, w.k, w.probes, w.t_q, w.vocab, cap, layers_per_call, overlap=overlap,
+                     fused=fused, vpool=vpool)
     chunk = lambda x: [x[:, lb:le].contiguous().cuda() for lb, le in path.chunks]
     out, H, fo = path.run(qs["q_emb"].cuda(), chunk(qs["q"]), chunk(qs["kq"]), chunk(qs["vq"]),
                           qs["logits"].cuda(), tau)
@@ -50,14 +51,14 @@ def _to_bf16_inputs(w, pool, qs):
     return w.scaled(dtype="bf16")
 
 
-def _check(w, nl, layers_per_call=None, tau=None, overlap=False, fused=False):
+def _check(w, nl, layers_per_call=None, tau=None, overlap=False, fused=False, vpool=False):
     pool, qs = wl.make_pool(w, n_layers=nl), wl.make_queries(w, n_layers=nl)
     if w.dtype == "fp32":     # the attention kernel is bf16: both sides get the same rounded inputs
         w = _to_bf16_inputs(w, pool, qs)
     H_want = orc.entropy(hp.f64(qs["logits"]))
     tau = float(np.median(H_want)) + 1e-2 if tau is None else tau
     sel, off, out_want, H_want, fo_want = oracle_path(w, pool, qs, nl, tau)
-    path, out = run_gpu_path(w, pool, qs, nl, tau, layers_per_call, overlap=overlap, fused=fused)
+    path, out = run_gpu_path(w, pool, qs, nl, tau, layers_per_call, overlap=overlap, fused=fused, vpool=vpool)
     assert np.array_equal(path.sel_idx.cpu().numpy(), sel)
     assert np.array_equal(path.ctx_off.cpu().numpy(), off)
     hp.assert_attn_close(out.cpu().double().numpy(), out_want, own_rounding=False)      # the stated bounds alone
@@ -96,6 +97,32 @@ def test_fused_variant_whole_path(cfg):
         w = wl.CONFIGS["cfg2"].scaled(n_shots=50, len_lo=1, len_hi=80, n_layers=2, batch=2, k=30, probes=(7, 30),
                                       t_q=150, head_dim=64, n_q_heads=6, n_kv_heads=3, vocab=2000, seed=35)
         _check(w, 2, fused=True)
+
+
+@pytest.mark.parametrize("cfg", ["cfg1", "8b", "d64"])
+def test_v_from_pool_variant_whole_path(cfg):
+    # K-only cache (gathered and re-encoded), V tiles copied from the pool inside attention: same oracle,
+    # same tolerances
+    if cfg == "cfg1":
+        _check(wl.CONFIGS["cfg1"], 1, vpool=True)
+    elif cfg == "8b":
+        w = wl.CONFIGS["cfg2"].scaled(n_shots=96, n_layers=3, batch=2, k=24, probes=(3, 6, 12, 24), t_q=48,
+                                      vocab=4000, seed=31)
+        _check(w, 3, layers_per_call=2, vpool=True)
+    else:
+        w = wl.CONFIGS["cfg2"].scaled(n_shots=50, len_lo=1, len_hi=80, n_layers=2, batch=2, k=30, probes=(7, 30),
+                                      t_q=150, head_dim=64, n_q_heads=6, n_kv_heads=3, vocab=2000, seed=35)
+        _check(w, 2, vpool=True)
+
+
+def test_v_from_pool_equals_the_full_cache_bit_for_bit():
+    # the same values reach the tensor cores in the same order: the two variants' outputs are identical
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=128, n_layers=2, batch=2, k=40, probes=(5, 13, 40), t_q=128, vocab=2000,
+                                  seed=39)
+    pool, qs = wl.make_pool(w, n_layers=2), wl.make_queries(w, n_layers=2)
+    _, out_full = run_gpu_path(w, pool, qs, 2, 5.0)
+    _, out_vpool = run_gpu_path(w, pool, qs, 2, 5.0, vpool=True)
+    assert torch.equal(out_full, out_vpool)
 
 
 def test_cuda_graph_replay_equals_the_plain_pass():

@@ -1,7 +1,8 @@
-"""Both attention variants on seeded random small shapes against the oracle: ragged shot
+"""The attention variants on seeded random small shapes against the oracle: ragged shot
 lengths down to one token, k = 1 and k = N, T_q = 1 and T_q just above a tile, head dims 64 and
 128, group sizes 1..8, nested probes, duplicated shot ids, several layers and queries.  Each case
-runs the materialised path (assemble + attention) and the fused path on the same inputs."""
+runs the materialised path (assemble + attention), the fused path and the V-from-pool path (K-only
+cache) on the same inputs."""
 import numpy as np
 import pytest
 import torch
@@ -55,6 +56,15 @@ def test_random_shape_both_variants(seed):
     ab.adapshot_query_attn_fused(model, dp, sel, off, cap, list(w.probes), q, kq, vq, 0, nl, out_f, None, ws, stf)
     torch.cuda.synchronize()
     assert stf.item() == 0
+    # K-only cache, V from the pool
+    out_v = torch.full_like(q, 9.0)
+    ws = torch.empty(max(ab.adapshot_attn_vpool_workspace_bytes(model, w.batch, len(w.probes), w.t_q, nl, cap), 256),
+                     dtype=torch.uint8, device="cuda")
+    stv = hp.new_status()
+    ab.adapshot_query_attn_vpool(model, dp, sel, kc, cap, off, list(w.probes), q, kq, vq, 0, nl, out_v, None, ws, stv)
+    torch.cuda.synchronize()
+    assert stv.item() == 0
+    assert torch.equal(out_v, out_m), "V from the pool must give the full cache's result bit for bit"
     # oracle (K' in fp64, never rounded)
     kp, vp = hp.f64(pool["k"][:nl]), hp.f64(pool["v"][:nl])
     for b in range(w.batch):
