@@ -226,7 +226,7 @@ ADAPSHOT_API int adapshot_query_attn_vpool(const adapshot_model_t* model, const 
  *   logits [R][row_stride] fp32 or bf16 (dtype), row_stride in elements, rows
  *   16-byte aligned; one pass with a running maximum, fp32 accumulation.
  *   Limits: R a multiple of rows_per_group, rows_per_group <= 8192, and
- *   R * splits < 2^31 with splits = min(ceil(296 / R), ceil(V / 4096)) (one CTA
+ *   R * splits < 2^31 with splits = min(ceil(1184 / R), ceil(V / 4096)) (one CTA
  *   per row and split); ADAPSHOT_ESHAPE otherwise.                              */
 ADAPSHOT_API size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V);
 ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V, int64_t row_stride,
@@ -257,7 +257,7 @@ ADAPSHOT_API int adapshot_entropy_subset(const void* logits, int32_t dtype, int3
  * and error codes as adapshot_entropy, minus `ws`: the per-split states live in
  * a fixed 192 KiB device array inside the library (one per GPU that loads it,
  * held until the process exits).
- *  - Limit: R * splits <= 16384 states, where splits = min(ceil(296 / R),
+ *  - Limit: R * splits <= 16384 states, where splits = min(ceil(1184 / R),
  *    ceil(V / 4096)); larger requests return ADAPSHOT_ECAPACITY and launch
  *    nothing.  (Examples within the limit: 8 rows x 128256; 224 rows x 128256.)
  *  - The first call on each device looks up the array's device address (with

@@ -78,9 +78,7 @@ entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride
   EntState st{-FLT_MAX, 0.f, 0.f};
 
   const int vec_end = begin + ((end - begin) / kVec) * kVec;   // slice is a multiple of kVec
-  for (int i = begin + threadIdx.x * kVec; i < vec_end; i += kEntThreads * kVec) {
-    float x[kVec];
-    uint4 raw = *reinterpret_cast<const uint4*>(row + i);
+  auto widen = [](const uint4& raw, float (&x)[kVec]) {
     if constexpr (sizeof(T) == 4) {
       x[0] = __uint_as_float(raw.x); x[1] = __uint_as_float(raw.y);
       x[2] = __uint_as_float(raw.z); x[3] = __uint_as_float(raw.w);
@@ -92,6 +90,26 @@ entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride
         x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
       }
     }
+  };
+  // four 16-byte loads in flight per thread: a CTA's 256 threads keep 16 KB on their way, which
+  // is what it takes to cover the DRAM latency at full bandwidth with a few CTAs per SM
+  constexpr int kUnroll = 4;
+  constexpr int kStep = kEntThreads * kVec;
+  int i = begin + threadIdx.x * kVec;
+  for (; i + (kUnroll - 1) * kStep < vec_end; i += kUnroll * kStep) {
+    uint4 raw[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) raw[u] = __ldcs(reinterpret_cast<const uint4*>(row + i + u * kStep));
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float x[kVec];
+      widen(raw[u], x);
+      ent_accumulate(st, x);
+    }
+  }
+  for (; i < vec_end; i += kStep) {
+    float x[kVec];
+    widen(__ldcs(reinterpret_cast<const uint4*>(row + i)), x);
     ent_accumulate(st, x);
   }
   for (int i = vec_end + threadIdx.x; i < end; i += kEntThreads) {   // ragged tail of the row
@@ -212,10 +230,11 @@ entropy_subset_finish_kernel(const float* __restrict__ partial, int n_split, int
 
 // A fixed figure rather than the SM count of the current device, so that the workspace size
 // can be asked for without a device and does not change from one GPU to another.
-constexpr int kEntTargetCtas = 296;
+constexpr int kEntTargetCtas = 1184;
 
 int ent_splits(int R, int V) {
-  // about kEntTargetCtas CTAs in all, each slice at least 4096 entries
+  // about kEntTargetCtas CTAs in all (one resident wave of 256-thread CTAs on 148 SMs), each slice
+  // at least 4096 entries
   int want = (kEntTargetCtas + R - 1) / R;
   int max_by_len = (V + 4095) / 4096;
   int s = want < max_by_len ? want : max_by_len;

@@ -66,7 +66,7 @@ def test_host_side_argument_checks_launch_nothing(ab):
                             kw.get("kc", fake), kw.get("vc", fake), kw.get("cap", 256), fake, kw.get("flags", 0), None, None]
     assert asm(*args(model, k=17)) == ab.ESHAPE
     assert asm(*args(model, le=2)) == ab.ESHAPE                       # layer range outside the model
-    assert asm(*args(model, flags=2)) == ab.EINVAL
+    assert asm(*args(model, flags=4)) == ab.EINVAL                    # an unknown flag
     assert asm(*args(model, vc=None)) == ab.EINVAL                    # only one of k_ctx / v_ctx
     assert asm(*args(model, kc=C.c_void_p(0x1008))) == ab.EALIGN
     bad = ab.make_model(1, 4, 1, 96, "fp32", 1e4)
