@@ -18,8 +18,12 @@ relative-position invariance of rotary attention.
 Parity status: every function here is pinned against closed forms and library
 routines.  entropy_subset (the two-token form of Eq. 2, outside the hot path)
 is pinned as arithmetic, but which of its two readings the paper means is not
-decidable from the text: for that choice it is "parity unpinned".  The
-attention-based relevance score of Eq. 5 is not implemented.
+decidable from the text: for that choice it is "parity unpinned".  The same
+holds for relevance_attention (Eq. 5): as printed, the softmax runs over one
+shot's own tokens, which makes every shot's mean score 1 / T_i; the function
+takes the one softmax over all pool keys instead and is pinned as arithmetic
+(brute force, closed forms, the printed form shown to be degenerate), while
+the choice of reading is "parity unpinned".
 
 Notation (paper, Sec. 3-4): N shots of lengths T_i, k selected shots, Hq/Hkv
 heads, G = Hq/Hkv, d head_dim, T_q query tokens, L_j context length of probe j.
@@ -85,6 +89,61 @@ def min_adjacent_gap(q_emb: np.ndarray, emb: np.ndarray, k: int) -> float:
         if gaps.size:
             best = min(best, float(gaps.min()))
     return best
+
+
+# --------------------------------------------------------------------------
+# Step 1, the paper's own selector (Sec. 4.2, Eq. 5 and the ranking sentence
+# after it): attention of the query's Q at a representative layer against the
+# cached K of every shot.  Eq. 5 as printed normalises over one shot's own
+# tokens, so every row of A^(i) sums to 1 and "the average over all tokens" is
+# 1 / T_i for every shot, whatever the query.  Reading taken: ONE softmax per
+# query token and head over the keys of the whole pool; a shot's relevance is
+# the attention mass that falls on its tokens, averaged over query tokens and
+# heads (per_token=True divides by T_i as well: the mean score of one of its
+# tokens).  Q and K enter as stored: no rotary rotation is applied here.
+# --------------------------------------------------------------------------
+def relevance_attention(q, k_layer, shot_off, per_token: bool = False, scale: float | None = None):
+    """s[i] for one query.  q [T_q, Hq, d]; k_layer [pool_tokens, Hkv, d] (the pool's K at the
+    representative layer); shot_off [N+1].  Query head h reads KV head h // G.  Returns fp64 [N];
+    without per_token the scores sum to 1."""
+    q = np.asarray(q, dtype=F64)
+    k = np.asarray(k_layer, dtype=F64)
+    so = np.asarray(shot_off, dtype=np.int64)
+    Tq, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    sc = (1.0 / np.sqrt(F64(d))) if scale is None else F64(scale)
+    N = so.shape[0] - 1
+    mass = np.zeros(N, dtype=F64)
+    for h in range(Hq):
+        logits = (q[:, h, :] @ k[:, h // G, :].T) * sc              # [T_q, pool_tokens]
+        m = logits.max(axis=1, keepdims=True)
+        e = np.exp(logits - m)
+        a = e / e.sum(axis=1, keepdims=True)                        # one softmax over the whole pool
+        for i in range(N):
+            mass[i] += a[:, so[i]:so[i + 1]].sum()
+    s = mass / F64(Tq * Hq)
+    if per_token:
+        s = s / (so[1:] - so[:-1]).astype(F64)
+    return s
+
+
+def select_topk_attention(q, k_layer, shot_off, k: int, per_token: bool = False, scale: float | None = None):
+    """Top-k by relevance_attention for a batch: q [B, T_q, Hq, d].  Ties -> lower shot id.
+    Returns (sel_idx int32 [B, k], score fp64 [B, k])."""
+    q = np.asarray(q, dtype=F64)
+    B = q.shape[0]
+    N = np.asarray(shot_off).shape[0] - 1
+    if not (1 <= k <= N):
+        raise ValueError("k must be in 1..N")
+    sel = np.empty((B, k), dtype=np.int32)
+    sc = np.empty((B, k), dtype=F64)
+    for b in range(B):
+        s = relevance_attention(q[b], k_layer, shot_off, per_token, scale)
+        order = np.argsort(-s, kind="stable")[:k]
+        sel[b] = order
+        sc[b] = s[order]
+    return sel, sc
 
 
 # --------------------------------------------------------------------------
@@ -217,6 +276,104 @@ def query_attn(q, kq, vq, k_ctx, v_ctx, L_list, base: float, scale: float | None
                 out[j, t, h] = o
                 lse[j, h, t] = l
     return out, lse
+
+
+# --------------------------------------------------------------------------
+# Step 4 in the paper's literal form (Sec. 4.1, "tree-structured attention"): ONE
+# sequence [shot_1 .. shot_n1, probe_1, shot_n1+1 .. shot_n2, probe_2, ...] and a
+# mask M.  The printed mask says which shots a probe sees; causality inside a
+# probe and the probe's view of its own tokens are added here as they must be for
+# the rows to equal Eq. 1 run alone.  Position ids: a shot keeps the position it
+# has in the plain concatenation of the shots (0 .. L-1, whatever probes are
+# interleaved), probe j's tokens sit at L_j + t.
+# --------------------------------------------------------------------------
+def tree_layout(ctx_off_row, probes, t_q: int):
+    """Token table of the interleaved sequence of one query.
+
+    ctx_off_row [k+1] offsets of the selected shots; probes ascending shot counts n_1 < ... < n_m.
+    Returns (kind [S] 0 = shot token / 1 = probe token, src [S] index into the assembled cache
+    (shot tokens) or j * t_q + t (probe tokens), pos [S] position ids, owner [S] shot slot r or
+    probe j, mask [S, S] bool: mask[i, c] = token i attends to token c)."""
+    off = np.asarray(ctx_off_row, dtype=np.int64)
+    kind, src, pos, owner = [], [], [], []
+    prev = 0
+    for j, n_j in enumerate(probes):
+        for r in range(prev, n_j):                      # the shots this probe adds
+            for p in range(int(off[r]), int(off[r + 1])):
+                kind.append(0); src.append(p); pos.append(p); owner.append(r)
+        L_j = int(off[n_j])
+        for t in range(t_q):
+            kind.append(1); src.append(j * t_q + t); pos.append(L_j + t); owner.append(j)
+        prev = n_j
+    kind, src, pos, owner = (np.asarray(a, dtype=np.int64) for a in (kind, src, pos, owner))
+    S = kind.shape[0]
+    mask = np.zeros((S, S), dtype=bool)
+    for i in range(S):
+        if kind[i] != 1:
+            continue                                    # shot tokens were prefilled alone: no row is computed
+        n_i = probes[int(owner[i])]
+        for c in range(S):
+            if kind[c] == 0:
+                mask[i, c] = owner[c] < n_i             # M_ij = 1 iff shot j is among the probe's first n_k
+            else:
+                mask[i, c] = owner[c] == owner[i] and src[c] <= src[i]    # its own tokens, causally
+    return kind, src, pos, owner, mask
+
+
+def masked_attention(q_rows, keys, vals, mask, scale: float):
+    """Dense attention with an explicit mask: out[i] = softmax_c(q_i . k_c * scale | mask[i, c]) . v_c.
+    q_rows [S, d], keys [S, d], vals [S, dv], mask [S, S]; rows without any visible key give zeros."""
+    q = np.asarray(q_rows, dtype=F64)
+    k = np.asarray(keys, dtype=F64)
+    v = np.asarray(vals, dtype=F64)
+    out = np.zeros((q.shape[0], v.shape[1]), dtype=F64)
+    for i in range(q.shape[0]):
+        vis = np.nonzero(mask[i])[0]
+        if vis.size == 0:
+            continue
+        s = (k[vis] @ q[i]) * scale
+        e = np.exp(s - s.max())
+        out[i] = (e / e.sum()) @ v[vis]
+    return out
+
+
+def tree_attention(q, kq, vq, k_ctx, v_ctx, ctx_off_row, probes, base: float, scale: float | None = None):
+    """All probe rows of one query at one layer through the single interleaved sequence and its
+    dense mask.  Arguments as query_attn (q [P, T_q, Hq, d], kq / vq [P, T_q, Hkv, d], k_ctx / v_ctx
+    [L, Hkv, d] assembled cache); returns out [P, T_q, Hq, d]."""
+    q = np.asarray(q, dtype=F64)
+    P, Tq, Hq, d = q.shape
+    Hkv = np.asarray(kq).shape[2]
+    G = Hq // Hkv
+    sc = (1.0 / np.sqrt(F64(d))) if scale is None else F64(scale)
+    kind, src, pos, owner, mask = tree_layout(ctx_off_row, probes, Tq)
+    is_probe = kind == 1
+    out = np.zeros((P, Tq, Hq, d), dtype=F64)
+    kq_flat = np.asarray(kq, dtype=F64).reshape(P * Tq, Hkv, d)
+    vq_flat = np.asarray(vq, dtype=F64).reshape(P * Tq, Hkv, d)
+    q_flat = q.reshape(P * Tq, Hq, d)
+    for h in range(Hq):
+        g = h // G
+        keys = np.zeros((kind.shape[0], d), dtype=F64)
+        vals = np.zeros((kind.shape[0], d), dtype=F64)
+        keys[~is_probe] = np.asarray(k_ctx, dtype=F64)[src[~is_probe], g]          # already at their positions
+        vals[~is_probe] = np.asarray(v_ctx, dtype=F64)[src[~is_probe], g]
+        keys[is_probe] = rope(kq_flat[src[is_probe], g], pos[is_probe].astype(F64), base)
+        vals[is_probe] = vq_flat[src[is_probe], g]
+        qr = np.zeros((kind.shape[0], d), dtype=F64)
+        qr[is_probe] = rope(q_flat[src[is_probe], h], pos[is_probe].astype(F64), base)
+        o = masked_attention(qr, keys, vals, mask, sc)
+        out[:, :, h, :] = o[is_probe].reshape(P, Tq, d)
+    return out
+
+
+def decode_row(q_new, k_own, v_own, k_ctx, v_ctx, L: int, kv_head: int, base: float, scale: float | None = None):
+    """One decode step after probing (Sec. 4.1: the chosen shots are "used for subsequent formal
+    inference"): the newest of T_own own tokens (query tokens plus what has been generated, at
+    positions L .. L+T_own-1) attends to the L context tokens of the chosen prefix and to all own
+    tokens.  q_new [d] un-rotated; k_own, v_own [T_own, Hkv, d] un-rotated.  Returns (out [d], lse)."""
+    T_own = np.asarray(k_own).shape[0]
+    return attn_row(q_new, k_own, v_own, k_ctx, v_ctx, L, T_own - 1, kv_head, base, scale)
 
 
 # --------------------------------------------------------------------------

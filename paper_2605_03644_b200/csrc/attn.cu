@@ -298,13 +298,14 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
 
 // Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
-// The fused variant's loader warps take the stages of tile i+1 before they hand over tile i,
-// which needs a third V stage; the room goes at the expense of the read-out staging.
+// The loader warps of the fused and V-from-pool variants work one tile ahead of the tile they hand
+// over (per-thread copies have the whole DRAM latency in front of them), which needs a third V
+// stage; the room goes at the expense of the read-out staging.
 template <int D, int MODE>
 struct AttnSmem {
   static constexpr int kKStages = 2;
-  static constexpr int kVStages = MODE == kModeFused ? 3 : 2;
-  static constexpr uint32_t kStageBytes = MODE == kModeFused ? 0 : 4096;  // per softmax warp: 32 rows x 128 bytes
+  static constexpr int kVStages = MODE != kModeCache ? 3 : 2;
+  static constexpr uint32_t kStageBytes = MODE != kModeCache ? 0 : 4096;  // per softmax warp: 32 rows x 128 bytes
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
   static constexpr uint32_t kOffQ = 0;                                    // Q of M tile A, then of M tile B
   static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
@@ -855,12 +856,10 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int i = 0; i < w.n_tiles; ++i, ++tv) {
           if ((tv & 1u) != par) continue;
           const uint32_t sv = tv % VS;
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag));
-          if (!ok) break;
           const bool own = i >= w.n_ctx;
           long long src_row[4];                 // source row (in rows of D elements) of tile rows lane + 32 q
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
+          for (int q4 = 0; q4 < 4; ++q4) {      // (looked up while the stage is still in use)
             const int row = lane + 32 * q4;
             if (!own) {
               const long long pos = (long long)(w.ctx_begin + i) * kTileN + row;
@@ -871,6 +870,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               src_row[q4] = t >= p.Tq ? -1 : ((long long)w.outer_own * p.Tq + t) * p.Hkv + w.g;
             }
           }
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag));
+          if (!ok) break;
           const __nv_bfloat16* vb = own ? p.vq : p.v_pool;
           const uint32_t v_base = base + SM::kOffV + sv * kTileBytes + col_off;
 #pragma unroll
@@ -1001,8 +1002,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           unsigned char* stg = base_ptr + SM::kOffStage + (warp - kSoftmaxWarp0) * SM::kStageBytes;
           const int sub = lane >> 3, ch = lane & 7;            // read-back: row 4 j + sub, chunk ch
           const int m0 = mt * kTileM + quarter * 32;
-          if constexpr (FUSED) {
-            // (no staging area in the fused variant's shared-memory plan: one row per thread)
+          if constexpr (MODE != kModeCache) {
+            // (no staging area in the shared-memory plan of the variants with loader warps: one row per thread)
             const int hq = w.g * p.G + m % p.G;
             __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t_row) * p.Hq) + hq) * (long long)D;
 #pragma unroll

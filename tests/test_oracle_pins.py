@@ -337,6 +337,143 @@ def test_min_adjacent_gap_on_hand_made_scores():
     assert orc.min_adjacent_gap(qe, np.array([[1.0, 1.0], [1.0, 1.0], [1.0, 1.0]]), 2) == np.inf
 
 
+# --------------------------------- literal tree layout (Sec. 4.1 mask equation)
+def test_tree_layout_hand_example():
+    # shots of 2, 1 and 3 tokens, probes after 1 and 3 shots, two probe tokens each:
+    # sequence  s0 s0 | p0 p0 | s1 s2 s2 s2 | p1 p1
+    off = np.array([0, 2, 3, 6])
+    kind, src, pos, owner, mask = orc.tree_layout(off, [1, 3], 2)
+    assert kind.tolist() == [0, 0, 1, 1, 0, 0, 0, 0, 1, 1]
+    assert src.tolist() == [0, 1, 0, 1, 2, 3, 4, 5, 2, 3]
+    assert pos.tolist() == [0, 1, 2, 3, 2, 3, 4, 5, 6, 7]          # shots keep 0..L-1; probe j sits at L_j + t
+    want = np.zeros((10, 10), dtype=int)
+    want[2, [0, 1, 2]] = 1                                          # probe 0, token 0: shot 0 and itself
+    want[3, [0, 1, 2, 3]] = 1
+    want[8, [0, 1, 4, 5, 6, 7, 8]] = 1                              # probe 1 sees all three shots, not probe 0
+    want[9, [0, 1, 4, 5, 6, 7, 8, 9]] = 1
+    assert np.array_equal(mask.astype(int), want)
+
+
+def test_tree_attention_equals_per_probe_attention_row_for_row():
+    rng = np.random.default_rng(41)
+    lens = np.array([3, 5, 2, 4, 1, 6])
+    so = np.concatenate([[0], np.cumsum(lens)])
+    Hq, Hkv, d, Tq, base = 4, 2, 8, 3, 10000.0
+    kp, vp = rng.standard_normal((1, int(so[-1]), Hkv, d)), rng.standard_normal((1, int(so[-1]), Hkv, d))
+    sel = np.array([4, 0, 5, 2, 1])
+    k_ctx, v_ctx, off = orc.assemble_kv(kp, vp, so, sel, base)
+    probes = [1, 2, 5]
+    q = rng.standard_normal((3, Tq, Hq, d))
+    kq, vq = rng.standard_normal((3, Tq, Hkv, d)), rng.standard_normal((3, Tq, Hkv, d))
+    tree = orc.tree_attention(q, kq, vq, k_ctx[0], v_ctx[0], off, probes, base)
+    per_probe, _ = orc.query_attn(q, kq, vq, k_ctx[0], v_ctx[0], [int(off[n]) for n in probes], base)
+    assert np.allclose(tree, per_probe, atol=1e-13)
+    # the mask matters: letting probe 0 see every shot changes its rows
+    full, _ = orc.query_attn(q, kq, vq, k_ctx[0], v_ctx[0], [int(off[5])] * 3, base)
+    assert np.abs(full[0] - tree[0]).max() > 1e-2
+
+
+def test_masked_attention_against_scipy():
+    rng = np.random.default_rng(42)
+    S, d = 7, 5
+    qm, km, vm = rng.standard_normal((S, d)), rng.standard_normal((S, d)), rng.standard_normal((S, 3))
+    mask = rng.random((S, S)) < 0.5
+    mask[2] = False                                                   # a row that sees nothing
+    got = orc.masked_attention(qm, km, vm, mask, 0.7)
+    for i in range(S):
+        if not mask[i].any():
+            assert np.all(got[i] == 0.0)
+            continue
+        logits = np.where(mask[i], (km @ qm[i]) * 0.7, -np.inf)
+        assert np.allclose(got[i], scipy.special.softmax(logits) @ vm, atol=1e-14)
+
+
+def test_decode_row_is_the_last_row_of_a_longer_probe():
+    rng = np.random.default_rng(43)
+    L, Hkv, d, T_own, base = 11, 2, 8, 5, 10000.0
+    k_ctx, v_ctx = rng.standard_normal((L + 4, Hkv, d)), rng.standard_normal((L + 4, Hkv, d))
+    k_own, v_own = rng.standard_normal((T_own, Hkv, d)), rng.standard_normal((T_own, Hkv, d))
+    qn = rng.standard_normal(d)
+    out, lse = orc.decode_row(qn, k_own, v_own, k_ctx, v_ctx, L, 1, base)
+    # the same through the dense definition: keys = context 0..L-1 and all own tokens at L..L+T_own-1
+    keys = np.concatenate([k_ctx[:L, 1], orc.rope(k_own[:, 1], L + np.arange(T_own, dtype=float), base)])
+    vals = np.concatenate([v_ctx[:L, 1], v_own[:, 1]])
+    s = keys @ orc.rope(qn, float(L + T_own - 1), base) / math.sqrt(d)
+    assert np.allclose(out, scipy.special.softmax(s) @ vals, atol=1e-14)
+    assert abs(lse - scipy.special.logsumexp(s)) < 1e-13
+
+
+# ------------------------------------- attention-based relevance (Eq. 5)
+def _tiny_relevance_case(seed=31):
+    rng = np.random.default_rng(seed)
+    lens = np.array([3, 1, 5, 2, 4])
+    so = np.concatenate([[0], np.cumsum(lens)])
+    Tq, Hq, Hkv, d = 4, 4, 2, 8
+    q = rng.standard_normal((Tq, Hq, d))
+    k = rng.standard_normal((int(so[-1]), Hkv, d))
+    return q, k, so, lens
+
+
+def test_relevance_attention_matches_python_loops_and_scipy():
+    q, k, so, lens = _tiny_relevance_case()
+    Tq, Hq, d = q.shape
+    G = Hq // k.shape[1]
+    want = np.zeros(len(lens))
+    for t in range(Tq):
+        for h in range(Hq):
+            logit = [sum(q[t, h, c] * k[j, h // G, c] for c in range(d)) / math.sqrt(d) for j in range(k.shape[0])]
+            a = scipy.special.softmax(np.array(logit))              # over ALL pool keys
+            for i in range(len(lens)):
+                want[i] += a[so[i]:so[i + 1]].sum()
+    want /= Tq * Hq
+    got = orc.relevance_attention(q, k, so)
+    assert np.allclose(got, want, atol=1e-14)
+    assert abs(got.sum() - 1.0) < 1e-13                             # the masses of all shots add up to one
+    assert np.allclose(orc.relevance_attention(q, k, so, per_token=True), want / lens, atol=1e-14)
+    # an explicit scale replaces 1 / sqrt(d)
+    assert np.allclose(orc.relevance_attention(q * 2.0, k, so, scale=0.5 / math.sqrt(d)), want, atol=1e-14)
+
+
+def test_relevance_attention_closed_forms():
+    q, k, so, lens = _tiny_relevance_case(32)
+    # identical keys everywhere: uniform attention, a shot's mass is its share of the pool's tokens
+    k_same = np.broadcast_to(k[:1], k.shape).copy()
+    assert np.allclose(orc.relevance_attention(q, k_same, so), lens / lens.sum(), atol=1e-14)
+    assert np.allclose(orc.relevance_attention(q, k_same, so, per_token=True), 1.0 / lens.sum(), atol=1e-15)
+    # zero queries: the same uniform distribution whatever the keys
+    assert np.allclose(orc.relevance_attention(q * 0.0, k, so), lens / lens.sum(), atol=1e-14)
+    # a shot whose keys point along the queries (large scores) takes nearly all of the mass and ranks first
+    qd = np.ones_like(q)
+    k2 = k * 0.01
+    k2[so[3]:so[4]] = 6.0
+    s = orc.relevance_attention(qd, k2, so)
+    assert s[3] > 0.999 and int(np.argmax(s)) == 3
+    sel, sc = orc.select_topk_attention(qd[None], k2, so, 2)
+    assert sel[0, 0] == 3 and sc[0, 0] == s[3]
+    # ties go to the lower shot id: shots 0 and 4 made of the same single key repeated, equal lengths
+    so_t = np.array([0, 2, 3, 5])
+    k_t = np.stack([k[0], k[0], k[1], k[0], k[0]])
+    sel, _ = orc.select_topk_attention(q[None], k_t, so_t, 3)
+    s_t = orc.relevance_attention(q, k_t, so_t)
+    assert s_t[0] == s_t[2] and list(sel[0]).index(0) < list(sel[0]).index(2)
+    # GQA: head h reads KV head h // G (expanding the KV heads changes nothing)
+    rep = np.repeat(k, q.shape[1] // k.shape[1], axis=1)
+    assert np.allclose(orc.relevance_attention(q, rep, so), orc.relevance_attention(q, k, so), atol=1e-15)
+
+
+def test_eq5_as_printed_is_degenerate():
+    # softmax over one shot's own tokens (Eq. 5 as printed): every row sums to one, so the mean over all
+    # entries of A^(i) is 1 / T_i for every query.  The reading taken must not behave like that.
+    q, k, so, lens = _tiny_relevance_case(33)
+    printed = []
+    for i in range(len(lens)):
+        logits = np.einsum("thd,jhd->htj", q[:, :2], k[so[i]:so[i + 1]]) / math.sqrt(q.shape[-1])
+        printed.append(scipy.special.softmax(logits, axis=-1).mean())
+    assert np.allclose(printed, 1.0 / lens, atol=1e-15)
+    got = orc.relevance_attention(q, k, so, per_token=True)
+    assert np.abs(got * lens.sum() - 1.0).max() > 0.05 and np.abs(got - 1.0 / lens).max() > 0.05
+
+
 # --------------------------------------------------------------- entropy
 def test_entropy_closed_forms_and_scipy():
     V = 1024
@@ -439,6 +576,10 @@ PIN_TESTS = [
     test_attention_closed_forms, test_attention_scale_is_inverse_sqrt_head_dim,
     test_gqa_head_mapping, test_cosine_against_scipy_and_python_sort,
     test_topk_ties_self_match_and_prefix_property, test_min_adjacent_gap_on_hand_made_scores,
+    test_tree_layout_hand_example, test_tree_attention_equals_per_probe_attention_row_for_row,
+    test_masked_attention_against_scipy, test_decode_row_is_the_last_row_of_a_longer_probe,
+    test_relevance_attention_matches_python_loops_and_scipy, test_relevance_attention_closed_forms,
+    test_eq5_as_printed_is_degenerate,
     test_entropy_closed_forms_and_scipy, test_threshold_rule_on_the_papers_case_study,
     test_subset_entropy_closed_forms_and_bounds, test_probe_rounds_on_the_papers_case_study,
 ]
@@ -520,6 +661,62 @@ def _mut_gap_stops_at_rank_k(q_emb, emb, k):
     return _ORIG["min_adjacent_gap"](q_emb, emb, k - 1) if k > 1 else np.inf
 
 
+def _mut_relevance_softmax_per_shot(q, k_layer, shot_off, per_token=False, scale=None):
+    # Eq. 5 as printed: the softmax normalises over one shot's own tokens
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k_layer, dtype=np.float64)
+    so = np.asarray(shot_off)
+    Tq, Hq, d = q.shape
+    G = Hq // k.shape[1]
+    sc = 1.0 / math.sqrt(d) if scale is None else scale
+    out = np.zeros(len(so) - 1)
+    for i in range(len(so) - 1):
+        for h in range(Hq):
+            a = scipy.special.softmax((q[:, h] @ k[so[i]:so[i + 1], h // G].T) * sc, axis=1)
+            out[i] += a.sum()
+    out /= Tq * Hq
+    return out / (so[1:] - so[:-1]) if per_token else out
+
+
+def _mut_relevance_no_scale(q, k_layer, shot_off, per_token=False, scale=None):
+    return _ORIG["relevance_attention"](q, k_layer, shot_off, per_token, 1.0 if scale is None else scale)
+
+
+def _mut_relevance_kv_head_zero(q, k_layer, shot_off, per_token=False, scale=None):
+    k = np.asarray(k_layer, dtype=np.float64)
+    return _ORIG["relevance_attention"](q, np.broadcast_to(k[:, :1], k.shape), shot_off, per_token, scale)
+
+
+def _mut_relevance_inclusive_segments(q, k_layer, shot_off, per_token=False, scale=None):
+    so = np.asarray(shot_off).copy()
+    so[1:-1] += 1                                               # shot boundaries off by one token
+    s = _ORIG["relevance_attention"](q, k_layer, so, False, scale)
+    return s / (np.asarray(shot_off)[1:] - np.asarray(shot_off)[:-1]) if per_token else s
+
+
+def _mut_tree_layout_probe_sees_earlier_probes(ctx_off_row, probes, t_q):
+    kind, src, pos, owner, mask = _ORIG["tree_layout"](ctx_off_row, probes, t_q)
+    mask = mask.copy()
+    for i in np.nonzero(kind == 1)[0]:
+        for c in np.nonzero(kind == 1)[0]:
+            if owner[c] < owner[i]:
+                mask[i, c] = True                                   # an earlier probe's tokens leak in
+    return kind, src, pos, owner, mask
+
+
+def _mut_tree_layout_positions_follow_the_sequence(ctx_off_row, probes, t_q):
+    kind, src, pos, owner, mask = _ORIG["tree_layout"](ctx_off_row, probes, t_q)
+    return kind, src, np.arange(kind.shape[0]), owner, mask        # position = index in the interleaved sequence
+
+
+def _mut_tree_layout_not_causal(ctx_off_row, probes, t_q):
+    kind, src, pos, owner, mask = _ORIG["tree_layout"](ctx_off_row, probes, t_q)
+    mask = mask.copy()
+    for i in np.nonzero(kind == 1)[0]:
+        mask[i, (kind == 1) & (owner == owner[i])] = True           # a probe token sees its later tokens
+    return kind, src, pos, owner, mask
+
+
 def _mut_first_ok_strict(H, tau, P):
     Hm = np.asarray(H).reshape(-1, P)
     return np.array([next((j for j in range(P) if Hm[b, j] > tau), -1)
@@ -582,6 +779,13 @@ _ORIG = {}
     ("min_adjacent_gap", _mut_gap_always_inf),
     ("min_adjacent_gap", _mut_gap_counts_ties),
     ("min_adjacent_gap", _mut_gap_stops_at_rank_k),
+    ("relevance_attention", _mut_relevance_softmax_per_shot),
+    ("relevance_attention", _mut_relevance_no_scale),
+    ("relevance_attention", _mut_relevance_kv_head_zero),
+    ("relevance_attention", _mut_relevance_inclusive_segments),
+    ("tree_layout", _mut_tree_layout_probe_sees_earlier_probes),
+    ("tree_layout", _mut_tree_layout_positions_follow_the_sequence),
+    ("tree_layout", _mut_tree_layout_not_causal),
     ("first_ok", _mut_first_ok_strict),
     ("probe_rounds", _mut_probe_rounds_lowest_entropy),
     ("probe_rounds", _mut_probe_rounds_runs_every_round),
@@ -593,7 +797,7 @@ _ORIG = {}
 ])
 def test_planted_mistakes_are_caught(name, mutant, monkeypatch):
     for n in ("rope", "plan_offsets", "entropy", "entropy_subset", "probe_rounds", "cosine_scores",
-              "min_adjacent_gap"):
+              "min_adjacent_gap", "relevance_attention", "tree_layout"):
         _ORIG[n] = getattr(orc, n)
     assert not _caught(), "pins must pass on the unmodified oracle"
     monkeypatch.setattr(orc, name, mutant)
