@@ -101,6 +101,29 @@ ADAPSHOT_API int adapshot_select(const adapshot_pool_t* pool, const float* q_emb
                     int32_t* sel_idx, float* sel_score,
                     void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
+/* ---- Step 1 with the paper's own relevance score (Sec. 4.2, Eq. 5 and the ranking sentence
+ * after it): attention of the query's Q at a representative layer against the cached K of every
+ * shot.  Eq. 5 as printed normalises over one shot's own tokens (every shot's mean score is then
+ * 1 / T_i, whatever the query); the reading taken is ONE softmax per query token and head over
+ * the keys of the whole pool at that layer:
+ *   a[t][h][j] = softmax_j( q[t][h] . k[layer][j][h / G] * scale ),  j over all pool tokens
+ *   s[b][i]    = (1 / (T_q Hq)) sum_{t,h} sum_{j in shot i} a[t][h][j]      (sums to 1 over i)
+ *   with ADAPSHOT_RELEVANCE_PER_TOKEN: s[b][i] / T_i (the mean score of one of its tokens).
+ * Q and K enter as stored (no rotary rotation is applied here); scale = model->softmax_scale
+ * or 1/sqrt(d).  sel_idx[b][r] = id of the r-th most relevant shot, equal scores by lower id.
+ *   q [B][T_q][Hq][d] bf16; sel_idx [B][k] int32 out; sel_score [B][k] fp32 out or NULL.
+ * bf16 tensor-core kernels (two passes over the layer's K: the normaliser, then the masses),
+ * fp32 exponentials, fp64 accumulation of the masses (by atomics: the last bits of a score may
+ * differ from run to run).  model->dtype must be ADAPSHOT_BF16; limits as adapshot_select,
+ * pool_tokens < 2^31 - 256.                                                                 */
+#define ADAPSHOT_RELEVANCE_PER_TOKEN 1u
+ADAPSHOT_API size_t adapshot_select_attn_workspace_bytes(const adapshot_model_t* model, const adapshot_pool_t* pool,
+                                            int32_t B, int32_t Tq, int32_t k);
+ADAPSHOT_API int adapshot_select_attn(const adapshot_model_t* model, const adapshot_pool_t* pool, int32_t layer,
+                         const void* q, int32_t B, int32_t Tq, int32_t k, uint32_t flags,
+                         int32_t* sel_idx, float* sel_score, void* ws, size_t ws_bytes,
+                         int32_t* status, void* stream);
+
 /* ---- Step 2: KV-level concatenation with position re-encoding (Sec. 4.3,
  * Eq. 7; offsets follow the two-shot example: a shot placed after r others
  * starts at the sum of their lengths).
@@ -217,6 +240,55 @@ ADAPSHOT_API int adapshot_query_attn_vpool(const adapshot_model_t* model, const 
                               const void* q, const void* kq, const void* vq, int32_t Tq,
                               int32_t layer_begin, int32_t layer_end, void* out, float* lse,
                               uint32_t flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* ---- Step 3 in the paper's literal form (Sec. 4.1, parallel multi-probe verification): ONE
+ * sequence [shot_1 .. shot_n1, probe_1, shot_n1+1 .. shot_n2, probe_2, ...] with the tree mask
+ * M_ij = 1 iff i is a token of probe_k and j belongs to its first n_k shots (plus, as causal
+ * attention requires, the probe's own earlier tokens).  The sequence is described by a segment
+ * table in HOST memory: seg_kind[i] is ADAPSHOT_SEG_SHOTS (seg_len[i] = number of selected
+ * shots in the run, taken in sel_idx order) or ADAPSHOT_SEG_PROBE (seg_len[i] = tokens of the
+ * probe).  Probes must each follow at least one new shot, have equal token counts, and the
+ * sequence must end with a probe; at most 16 probes (ADAPSHOT_ESHAPE otherwise).  The shots'
+ * K/V come from the assembled cache, so the tensors hold the probe tokens only, in sequence
+ * order: q_seq [B][nl][N_probe_tokens][Hq][d], kq_seq / vq_seq [..][Hkv][d], out_seq like
+ * q_seq.  No dense mask is materialised: a probe's row range of visible keys follows from the
+ * table.  Position ids (shots keep 0 .. L-1 of their plain concatenation, token t of probe k
+ * sits at L_k + t) are written to pos_seq [B][N_probe_tokens] int64 when it is not NULL.
+ * adapshot_tree_layout is the table's parser alone (host only; probe_nshots [16] out).
+ * Everything else as adapshot_query_attn.                                                  */
+#define ADAPSHOT_SEG_SHOTS 0
+#define ADAPSHOT_SEG_PROBE 1
+ADAPSHOT_API int adapshot_tree_layout(const int32_t* seg_kind, const int32_t* seg_len, int32_t n_seg, int32_t k,
+                         int32_t* probe_nshots, int32_t* P_out, int32_t* Tq_out);
+ADAPSHOT_API int adapshot_tree_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx,
+                       int64_t ctx_cap, const int64_t* ctx_off, int32_t B, int32_t k,
+                       const int32_t* seg_kind, const int32_t* seg_len, int32_t n_seg,
+                       const void* q_seq, const void* kq_seq, const void* vq_seq,
+                       int32_t layer_begin, int32_t layer_end, void* out_seq, float* lse,
+                       int64_t* pos_seq, uint32_t flags, void* ws, size_t ws_bytes, int32_t* status,
+                       void* stream);
+
+/* ---- Decoding over the chosen prefix (Sec. 4.1: the shot count that met the threshold is
+ * "used for subsequent formal inference").  Query b continues over its first n_shots[b]
+ * selected shots (context length L_b = ctx_off[b][n_shots[b]]) with T_own own tokens (its
+ * query tokens and whatever has been generated so far) at positions L_b .. L_b + T_own - 1;
+ * the call computes the rows of the LAST T_new of them (T_new = 1: one decode step; T_new =
+ * T_own: the prefill of the query over the chosen prefix).  Row t sees the L_b context tokens
+ * and the own tokens up to its own.
+ *   n_shots : DEVICE int32 [B], 1 <= n_shots[b] <= k (e.g. derived from first_ok); a value
+ *             outside that range is reported as ADAPSHOT_EINDEX in `status` and clamped
+ *   q_new   : [B][nl][T_new][Hq][d];  k_own, v_own : [B][nl][T_own][Hkv][d]  (un-rotated)
+ *   out     : [B][nl][T_new][Hq][d];  lse [B][nl][Hq][T_new] or NULL
+ * Same kernels as adapshot_query_attn (a decode step is bound by the K/V bytes it reads, not
+ * by the tensor cores); limits: B <= 256, T_own >= T_new >= 1.                              */
+ADAPSHOT_API size_t adapshot_decode_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t T_new,
+                                       int32_t T_own, int32_t n_layers_in_call);
+ADAPSHOT_API int adapshot_decode_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx,
+                         int64_t ctx_cap, const int64_t* ctx_off, int32_t B, int32_t k,
+                         const int32_t* n_shots, const void* q_new, const void* k_own, const void* v_own,
+                         int32_t T_new, int32_t T_own, int32_t layer_begin, int32_t layer_end,
+                         void* out, float* lse, uint32_t flags, void* ws, size_t ws_bytes,
+                         int32_t* status, void* stream);
 
 /* ---- Step 4: confidence probe (Eq. 2 over the whole vocabulary, natural log)
  * and the threshold rule that follows it.

@@ -26,10 +26,12 @@ ASSEMBLE_KEEP_PLAN = 1
 ASSEMBLE_K_ONLY = 2
 
 EXPORTS = [
-    "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_assemble_kv", "adapshot_assemble_kv_from",
+    "adapshot_select_workspace_bytes", "adapshot_select", "adapshot_select_attn_workspace_bytes",
+    "adapshot_select_attn", "adapshot_assemble_kv", "adapshot_assemble_kv_from",
     "adapshot_attn_workspace_bytes", "adapshot_query_attn",
     "adapshot_attn_fused_workspace_bytes", "adapshot_query_attn_fused",
     "adapshot_attn_vpool_workspace_bytes", "adapshot_query_attn_vpool",
+    "adapshot_tree_layout", "adapshot_tree_attn", "adapshot_decode_workspace_bytes", "adapshot_decode_attn",
     "adapshot_entropy_workspace_bytes", "adapshot_entropy", "adapshot_entropy_subset",
     "adapshot_entropy_static",
     "adapshot_profile", "adapshot_profile_attn_main_ms", "adapshot_selftest_wait_timeout",
@@ -58,6 +60,12 @@ def _sig(name, restype, argtypes):
 _vp, _i32, _i64, _sz, _u32, _f = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t, C.c_uint32, C.c_float
 _select_ws = _sig("adapshot_select_workspace_bytes", _sz, [_i32, _i32, _i32])
 _select = _sig("adapshot_select", C.c_int, [C.POINTER(PoolT), _vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp, _vp])
+_select_attn_ws = _sig("adapshot_select_attn_workspace_bytes", _sz,
+                       [C.POINTER(ModelT), C.POINTER(PoolT), _i32, _i32, _i32])
+_select_attn = _sig("adapshot_select_attn", C.c_int,
+                    [C.POINTER(ModelT), C.POINTER(PoolT), _i32, _vp, _i32, _i32, _i32, _u32, _vp, _vp, _vp, _sz,
+                     _vp, _vp])
+RELEVANCE_PER_TOKEN = 1
 _assemble = _sig("adapshot_assemble_kv", C.c_int,
                  [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _i32, _i32, _i32, _i32, _vp, _vp, _i64,
                   _vp, _u32, _vp, _vp])
@@ -91,6 +99,18 @@ _attn_vpool_ws = _sig("adapshot_attn_vpool_workspace_bytes", _sz,
 _attn_vpool = _sig("adapshot_query_attn_vpool", C.c_int,
                    [C.POINTER(ModelT), C.POINTER(PoolT), _vp, _vp, _i64, _vp, _i32, _i32, C.POINTER(_i32), _i32,
                     _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+
+
+_tree_layout = _sig("adapshot_tree_layout", C.c_int,
+                    [C.POINTER(_i32), C.POINTER(_i32), _i32, _i32, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)])
+_tree_attn = _sig("adapshot_tree_attn", C.c_int,
+                  [C.POINTER(ModelT), _vp, _vp, _i64, _vp, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32), _i32,
+                   _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+_decode_ws = _sig("adapshot_decode_workspace_bytes", _sz, [C.POINTER(ModelT), _i32, _i32, _i32, _i32])
+_decode = _sig("adapshot_decode_attn", C.c_int,
+               [C.POINTER(ModelT), _vp, _vp, _i64, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
+                _vp, _vp, _u32, _vp, _sz, _vp, _vp])
+SEG_SHOTS, SEG_PROBE = 0, 1
 
 
 _profile = _sig("adapshot_profile", C.c_int, [C.c_int])
@@ -173,6 +193,20 @@ def adapshot_select(pool: Pool, q_emb: torch.Tensor, k: int, sel_idx: torch.Tens
                    _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
 
 
+def adapshot_select_attn_workspace_bytes(model: ModelT, pool: Pool, B: int, Tq: int, k: int) -> int:
+    return _select_attn_ws(C.byref(model), C.byref(pool.c), B, Tq, k)
+
+
+def adapshot_select_attn(model: ModelT, pool: Pool, layer: int, q: torch.Tensor, k: int, sel_idx: torch.Tensor,
+                         sel_score: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor,
+                         per_token: bool = False):
+    """Top-k by attention mass (Sec. 4.2): q [B][T_q][Hq][d] bf16 against the pool's K at `layer`."""
+    B, Tq = q.shape[0], q.shape[1]
+    _check(_select_attn(C.byref(model), C.byref(pool.c), layer, _ptr(q), B, Tq, k,
+                        RELEVANCE_PER_TOKEN if per_token else 0, _ptr(sel_idx), _ptr(sel_score), _ptr(ws),
+                        ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
 def adapshot_assemble_kv(model: ModelT, pool: Pool, sel_idx: torch.Tensor, layer_begin: int,
                          layer_end: int, k_ctx: Optional[torch.Tensor], v_ctx: Optional[torch.Tensor],
                          ctx_cap: int, ctx_off: torch.Tensor, status: torch.Tensor, flags: int = 0):
@@ -246,6 +280,52 @@ def adapshot_query_attn_vpool(model: ModelT, pool: Pool, sel_idx: torch.Tensor, 
     _check(_attn_vpool(C.byref(model), C.byref(pool.c), _ptr(sel_idx), _ptr(k_ctx), ctx_cap, _ptr(ctx_off), B, k,
                        arr, P, _ptr(q), _ptr(kq), _ptr(vq), Tq, layer_begin, layer_end, _ptr(out), _ptr(lse),
                        flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def _seg_arrays(segments):
+    n = len(segments)
+    kinds = (_i32 * n)(*[int(kd) for kd, _ in segments])
+    lens = (_i32 * n)(*[int(ln) for _, ln in segments])
+    return kinds, lens, n
+
+
+def adapshot_tree_layout(segments, k: int):
+    """Parses a segment table [(SEG_SHOTS, n shots) | (SEG_PROBE, tokens), ...] of the interleaved
+    sequence; returns (probe shot counts, tokens per probe)."""
+    kinds, lens, n = _seg_arrays(segments)
+    probes = (_i32 * 16)()
+    P, Tq = _i32(0), _i32(0)
+    _check(_tree_layout(kinds, lens, n, k, probes, C.byref(P), C.byref(Tq)))
+    return [int(probes[i]) for i in range(P.value)], int(Tq.value)
+
+
+def adapshot_tree_attn(model: ModelT, k_ctx: torch.Tensor, v_ctx: torch.Tensor, ctx_cap: int,
+                       ctx_off: torch.Tensor, k: int, segments, q_seq: torch.Tensor, kq_seq: torch.Tensor,
+                       vq_seq: torch.Tensor, layer_begin: int, layer_end: int, out_seq: torch.Tensor,
+                       lse: Optional[torch.Tensor], pos_seq: Optional[torch.Tensor], ws: torch.Tensor,
+                       status: torch.Tensor, flags: int = 0):
+    B = q_seq.shape[0]
+    kinds, lens, n = _seg_arrays(segments)
+    _check(_tree_attn(C.byref(model), _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), B, k, kinds, lens, n,
+                      _ptr(q_seq), _ptr(kq_seq), _ptr(vq_seq), layer_begin, layer_end, _ptr(out_seq), _ptr(lse),
+                      _ptr(pos_seq), flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
+
+
+def adapshot_decode_workspace_bytes(model: ModelT, B: int, T_new: int, T_own: int, n_layers_in_call: int) -> int:
+    return _decode_ws(C.byref(model), B, T_new, T_own, n_layers_in_call)
+
+
+def adapshot_decode_attn(model: ModelT, k_ctx: torch.Tensor, v_ctx: torch.Tensor, ctx_cap: int,
+                         ctx_off: torch.Tensor, k: int, n_shots: torch.Tensor, q_new: torch.Tensor,
+                         k_own: torch.Tensor, v_own: torch.Tensor, layer_begin: int, layer_end: int,
+                         out: torch.Tensor, lse: Optional[torch.Tensor], ws: torch.Tensor, status: torch.Tensor,
+                         flags: int = 0):
+    B, T_new, T_own = q_new.shape[0], q_new.shape[2], k_own.shape[2]
+    if n_shots.dtype != torch.int32:
+        raise ValueError("n_shots must be int32")
+    _check(_decode(C.byref(model), _ptr(k_ctx), _ptr(v_ctx), ctx_cap, _ptr(ctx_off), B, k, _ptr(n_shots),
+                   _ptr(q_new), _ptr(k_own), _ptr(v_own), T_new, T_own, layer_begin, layer_end, _ptr(out),
+                   _ptr(lse), flags, _ptr(ws), ws.numel() * ws.element_size(), _ptr(status), _stream()))
 
 
 def adapshot_entropy_workspace_bytes(R: int, V: int) -> int:

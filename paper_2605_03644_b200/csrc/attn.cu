@@ -31,6 +31,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "tma_host.cuh"
 
 namespace {
 
@@ -44,7 +45,8 @@ constexpr int kUnitCost = 4;          // fixed cost of starting a unit, in tiles
 constexpr int kTileM = 128;          // query rows per M tile (TMEM lanes)
 constexpr int kTileN = 128;          // keys per tile
 constexpr int kAttnThreads = 320;    // warp 0 TMA, warp 1 MMA, warps 2-5 softmax A, warps 6-9 softmax B
-constexpr int kFusedThreads = 384;   // fused / V-from-pool variants: warps 2-3 are loaders, softmax on warps 4-11
+constexpr int kFusedThreads = 384;   // fused variant: warps 2-3 load and rotate K/V, softmax on warps 4-11
+constexpr int kVPoolThreads = 352;   // V-from-pool variant: the cache variant's warps plus warp 10, which gathers V
 constexpr int kModeCache = 0;        // K and V tiles by TMA from the assembled cache
 constexpr int kModeFused = 1;        // K and V tiles from the pool, K re-encoded in shared memory
 constexpr int kModeVPool = 2;        // K tiles by TMA from a K-only cache, V tiles from the pool
@@ -78,12 +80,13 @@ struct AttnParams {
   float* lse;                 // [B][nl][P][Hq][Tq] or null
   int32_t* status;
   int B, P, Tq, Hq, Hkv, G, nl;
+  int To;                     // own tokens per probe (>= Tq): the Tq rows are the last Tq of them
   int n_mt, n_mp, gang, n_gangs;
   float scale_log2;           // softmax_scale * log2(e)
   // fused variant only: K/V tiles come from the pool (and from the probe's own rotated keys)
   const __nv_bfloat16* k_pool;   // [n_layers][pool_tokens][Hkv][D]
   const __nv_bfloat16* v_pool;
-  const __nv_bfloat16* kq_rot;   // [B*nl*P][Tq][Hkv][D], rotated by the prep kernel
+  const __nv_bfloat16* kq_rot;   // [B*nl*P][To][Hkv][D], rotated by the prep kernel
   const __nv_bfloat16* vq;
   const int* row_map;            // [B][ctx_cap]: pool token of every context position, -1 beyond L
   const int* off_map;            // [B][ctx_cap]: first position of the shot a position lies in (k_pos_mode 1)
@@ -96,13 +99,16 @@ struct AttnParams {
 
 struct PrepParams {
   const __nv_bfloat16* q;     // [B][nl][P][Tq][Hq][D]
-  const __nv_bfloat16* kq;    // [B][nl][P][Tq][Hkv][D]
+  const __nv_bfloat16* kq;    // [B][nl][P][To][Hkv][D]
   __nv_bfloat16* q_rot;       // [B*nl*P*Hkv][Tq*G][D]
   __nv_bfloat16* kq_rot;      // layout of kq
   const long long* ctx_off;
   Sched* sched;
   long long ctx_cap;
   int B, k, P, Tq, Hq, Hkv, nl, n_gangs;
+  int To;                     // own tokens per probe: the Tq query rows are the last Tq of them
+  const int* nshots_dev;      // per-query shot count of the (single) probe, device memory, or null
+  int32_t* status;
   double rope_base;
   double theta[64];           // theta_i = rope_base^(-2i/D), formed on the host
   int nshots[kMaxProbes];
@@ -132,6 +138,18 @@ __device__ __forceinline__ uint4 bf16x8_pack(const float* x) {
 
 constexpr int kPrepParts = 4;
 
+// Shots of probe j of query b: from the host list, or (decode over the prefix each query chose)
+// from a per-query device array; a count outside 1..k is reported and clamped.
+__device__ __forceinline__ int probe_shots(const PrepParams& p, int b, int j) {
+  if (p.nshots_dev == nullptr) return p.nshots[j];
+  int n = p.nshots_dev[b];
+  if (n < 1 || n > p.k) {
+    ads_set_status(p.status, ADAPSHOT_EINDEX);
+    n = n < 1 ? 1 : p.k;
+  }
+  return n;
+}
+
 // kPrepParts warps per probe token (b, l, j, t): all Hq query heads and Hkv key heads of the
 // token rotate by the same angles (L_j + t) * theta_i.  The last block writes the schedule instead.
 template <int D>
@@ -146,11 +164,11 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
     __shared__ int s_nsu[kMaxPairs];
     Sched* sc = p.sched;
     const int n_pairs = p.P * p.B;
-    const int n_own = (p.Tq + kTileN - 1) / kTileN;
+    const int n_own = (p.To + kTileN - 1) / kTileN;
     const long long units_per_pair = (long long)p.nl * p.Hkv;
     for (int pi = threadIdx.x; pi < n_pairs; pi += blockDim.x) {
       const int j = p.P - 1 - pi / p.B, b = pi % p.B;
-      long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
+      long long Lj = p.ctx_off[(long long)b * (p.k + 1) + probe_shots(p, b, j)];
       Lj = Lj > p.ctx_cap ? p.ctx_cap : (Lj < 0 ? 0 : Lj);
       const int n_ctx = (int)((Lj + kTileN - 1) / kTileN);
       sc->Lj[pi] = Lj;
@@ -199,17 +217,19 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
     return;
   }
   const long long gw = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long tok = gw / kPrepParts;            // kPrepParts warps share the heads of one token
+  const long long tok = gw / kPrepParts;            // kPrepParts warps share the heads of one own token
   const int part = (int)(gw % kPrepParts);
-  const long long n_tok = (long long)p.B * p.nl * p.P * p.Tq;
+  const long long n_tok = (long long)p.B * p.nl * p.P * p.To;
   if (tok >= n_tok) return;
-  const int t = (int)(tok % p.Tq);
-  const long long bpj = tok / p.Tq;                 // (b*nl + l)*P + j
+  const int u_own = (int)(tok % p.To);              // own token u sits at position L_j + u
+  const long long bpj = tok / p.To;                 // (b*nl + l)*P + j
   const int j = (int)(bpj % p.P);
   const int b = (int)(bpj / ((long long)p.P * p.nl));
-  const long long Lj = p.ctx_off[(long long)b * (p.k + 1) + p.nshots[j]];
-  const double pos = (double)(Lj + t);
+  const long long Lj = p.ctx_off[(long long)b * (p.k + 1) + probe_shots(p, b, j)];
+  const double pos = (double)(Lj + u_own);
   const int G = p.Hq / p.Hkv;
+  const int t = u_own - (p.To - p.Tq);              // query row of this token (the last Tq own tokens have one)
+  const bool has_q = t >= 0;
 
   const int jcol = lane % HALF_V;
   float sn[8], cs[8];
@@ -217,7 +237,7 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   for (int e = 0; e < 8; ++e) {
     rope_sincos(pos, p.theta[jcol * 8 + e], &sn[e], &cs[e]);
   }
-  const uint4* qsrc = reinterpret_cast<const uint4*>(p.q) + tok * p.Hq * VPH;
+  const uint4* qsrc = reinterpret_cast<const uint4*>(p.q) + (bpj * p.Tq + (has_q ? t : 0)) * p.Hq * VPH;
   const uint4* ksrc = reinterpret_cast<const uint4*>(p.kq) + tok * p.Hkv * VPH;
   uint4* kdst = reinterpret_cast<uint4*>(p.kq_rot) + tok * p.Hkv * VPH;
   uint4* qdst_base = reinterpret_cast<uint4*>(p.q_rot);
@@ -225,6 +245,7 @@ __global__ void __launch_bounds__(256) attn_prep_kernel(const PrepParams p) {
   for (int u = part * 32 + lane; u < units; u += 32 * kPrepParts) {
     const int head = u / HALF_V;                    // column == jcol since 32 % HALF_V == 0
     const bool is_q = head < p.Hq;
+    if (is_q && !has_q) continue;
     const uint4* src = is_q ? qsrc + head * VPH + jcol : ksrc + (head - p.Hq) * VPH + jcol;
     float x[8], y[8], xr[8], yr[8];
     bf16x8_unpack(src[0], x);
@@ -298,14 +319,13 @@ __global__ void __launch_bounds__(256) attn_fused_plan_kernel(const FusedPlanPar
 
 // Shared-memory plan.  Every operand tile is made of [128 rows][128 bytes] sub-tiles
 // written by TMA with the 128-byte swizzle; D = 128 needs two of them per tile.
-// The loader warps of the fused and V-from-pool variants work one tile ahead of the tile they hand
-// over (per-thread copies have the whole DRAM latency in front of them), which needs a third V
-// stage; the room goes at the expense of the read-out staging.
+// The fused variant's loader warps take the stages of tile i+1 before they hand over tile i,
+// which needs a third V stage; the room goes at the expense of the read-out staging.
 template <int D, int MODE>
 struct AttnSmem {
   static constexpr int kKStages = 2;
-  static constexpr int kVStages = MODE != kModeCache ? 3 : 2;
-  static constexpr uint32_t kStageBytes = MODE != kModeCache ? 0 : 4096;  // per softmax warp: 32 rows x 128 bytes
+  static constexpr int kVStages = MODE == kModeFused ? 3 : 2;
+  static constexpr uint32_t kStageBytes = MODE == kModeFused ? 0 : 4096;  // per softmax warp: 32 rows x 128 bytes
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
   static constexpr uint32_t kOffQ = 0;                                    // Q of M tile A, then of M tile B
   static constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
@@ -418,7 +438,7 @@ __device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, 
   w.n_ctx = max(0, ctx_end - pc.t0);
   // own-token tiles this M pair can see (causal): tokens up to the pair's last row
   const int row_hi = min(p.Tq * p.G - 1, mp * 2 * kTileM + 2 * kTileM - 1);
-  const int own_need = (row_hi / p.G) / kTileN + 1;
+  const int own_need = (p.To - p.Tq + row_hi / p.G) / kTileN + 1;
   w.own_begin = max(pc.t0, pc.n_ctx) - pc.n_ctx;
   const int own_end = min(pc.t1 - pc.n_ctx, own_need);
   w.n_own = max(0, own_end - w.own_begin);
@@ -435,7 +455,7 @@ __device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, 
 // copies into the swizzled tile layout) and K is rotated in shared memory by two loader warps,
 // so that no re-encoded cache is ever written to HBM; TMA then only brings Q.
 template <int D, int MODE>
-__global__ void __launch_bounds__(MODE != kModeCache ? kFusedThreads : kAttnThreads, 1)
+__global__ void __launch_bounds__(MODE == kModeFused ? kFusedThreads : (MODE == kModeVPool ? kVPoolThreads : kAttnThreads), 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
                  const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
@@ -448,7 +468,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, 0);
   constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, 1);
   constexpr uint32_t kTmemS = 0, kTmemO = 256;
-  constexpr int kSoftmaxWarp0 = MODE != kModeCache ? 4 : 2;   // first of the eight softmax warps
+  constexpr int kSoftmaxWarp0 = FUSED ? 4 : 2;          // first of the eight softmax warps
+  constexpr int kGatherWarp = kSoftmaxWarp0 + 8;        // V-from-pool variant: the warp that gathers the V tiles
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -476,7 +497,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int i = 0; i < 3; ++i) {
       mbar_init(bar(kBarKFull + i), FUSED ? kLoaders : 1);
       mbar_init(bar(kBarKEmpty + i), 1);
-      mbar_init(bar(kBarVFull + i), FUSED ? kLoaders : (VPOOL ? 32 : 1));
+      mbar_init(bar(kBarVFull + i), FUSED ? kLoaders : 1);
       mbar_init(bar(kBarVEmpty + i), 1);
     }
     mbar_init(bar(kBarDrain), 1);
@@ -729,7 +750,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           src[u] = r < 0 ? -1 : (((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g) * D;
         } else {
           const int t = (w.own_begin + i - w.n_ctx) * kTileN + row;
-          src[u] = t >= p.Tq ? -1 : (((long long)w.outer_own * p.Tq + t) * p.Hkv + w.g) * D;
+          src[u] = t >= p.To ? -1 : (((long long)w.outer_own * p.To + t) * p.Hkv + w.g) * D;
         }
       }
       const __nv_bfloat16* kb = own ? p.kq_rot : p.k_pool;
@@ -830,64 +851,60 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
     cp_async_wait<0>();
-  } else if (VPOOL && warp < 4) {
-    // --------------------------------------- loader: V tiles straight from the pool
-    // Eq. 7 corrects K only, so V needs no assembled copy: the tile's 128 context positions are
-    // looked up in the row map and their rows copied from the pool by per-thread async copies
-    // (zero fill beyond the context) into the swizzled layout the PV descriptors expect.  Warp 2
-    // serves the even tiles of the CTA's tile sequence, warp 3 the odd ones, each with one tile in
-    // flight; a lane copies the same 16-byte column of CPR-spaced rows, so a warp instruction
-    // reads whole 128- or 256-byte rows.
-    constexpr int CPR = D / 8;                 // 16-byte chunks per row
-    constexpr int RPI = 32 / CPR;              // rows per warp instruction
-    constexpr int NU = kTileN / RPI;           // copies per lane and tile
-    const uint32_t par = (uint32_t)(warp - 2);
-    const int c = lane % CPR, rsub = lane / CPR;
-    const uint32_t col_off = (uint32_t)(c / 8) * 16384u;
-    const int j = c & 7;
+  } else if (VPOOL && warp == kGatherWarp) {
+    // ----------------------------------------- V tiles straight from the pool (TMA row gather)
+    // Eq. 7 corrects K only, so V needs no assembled copy: the 128 context positions of a tile are
+    // looked up in the row map and their pool rows fetched four at a time by TMA gather copies
+    // (one-row boxes of a 2-D map over all V rows of the pool, 128-byte swizzle, so the tile lands
+    // in the layout the PV descriptors expect).  Lane i brings rows 4 i .. 4 i + 3; rows beyond the
+    // context (their P is exactly zero) read some valid row instead of being skipped, so that every
+    // tile delivers the same number of bytes to its barrier.
     uint32_t tv = 0;
     bool ok = true;
     Walker wk = wk0;
     Piece pc;
+    if (lane == 0) { tma_prefetch_desc(&tm_vctx); tma_prefetch_desc(&tm_vown); }
     while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
       for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
         Item w;
         make_item(p, pc, gang_id, mp, w);
         for (int i = 0; i < w.n_tiles; ++i, ++tv) {
-          if ((tv & 1u) != par) continue;
           const uint32_t sv = tv % VS;
           const bool own = i >= w.n_ctx;
-          long long src_row[4];                 // source row (in rows of D elements) of tile rows lane + 32 q
+          int y[4];                                    // rows of the 2-D V map (in rows of D elements)
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {      // (looked up while the stage is still in use)
-            const int row = lane + 32 * q4;
+          for (int q4 = 0; q4 < 4; ++q4) {             // (looked up while the stage may still be in use)
+            const int row = 4 * lane + q4;
             if (!own) {
               const long long pos = (long long)(w.ctx_begin + i) * kTileN + row;
-              const int r = pos < p.ctx_cap ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
-              src_row[q4] = r < 0 ? -1 : ((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g;
+              int r = pos < p.ctx_cap ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
+              if (r < 0) r = 0;
+              y[q4] = (int)(((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g);
             } else {
-              const int t = (w.own_begin + i - w.n_ctx) * kTileN + row;
-              src_row[q4] = t >= p.Tq ? -1 : ((long long)w.outer_own * p.Tq + t) * p.Hkv + w.g;
+              const int t = min((w.own_begin + i - w.n_ctx) * kTileN + row, p.To - 1);
+              y[q4] = (int)(((long long)w.outer_own * p.To + t) * p.Hkv + w.g);
             }
           }
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag));
-          if (!ok) break;
-          const __nv_bfloat16* vb = own ? p.vq : p.v_pool;
-          const uint32_t v_base = base + SM::kOffV + sv * kTileBytes + col_off;
-#pragma unroll
-          for (int u = 0; u < NU; ++u) {
-            const int row = u * RPI + rsub;
-            const long long sr = __shfl_sync(0xffffffffu, src_row[(u * RPI) / 32], row & 31);
-            const __nv_bfloat16* g = vb + (sr < 0 ? 0 : sr) * D + c * 8;
-            cp_async16(v_base + row * 128u + ((uint32_t)(j ^ (row & 7)) << 4), g, sr < 0 ? 0u : 16u);
+          if (lane == 0) {
+            ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
+            if (ok) mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
           }
-          cp_async_commit();
-          cp_async_wait<0>();
-          fence_proxy_async_smem();
-          mbar_arrive(bar(kBarVFull + sv));
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
+          const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
+          const uint32_t dst = base + SM::kOffV + sv * kTileBytes + (uint32_t)(4 * lane) * 128u;
+#pragma unroll
+          for (int s2 = 0; s2 < SUB; ++s2)
+            tma_gather4(dst + s2 * 16384u, mv, bar(kBarVFull + sv), s2 * 64, y[0], y[1], y[2], y[3]);
         }
       }
     }
+    if (!ok && lane == 0) {
+      // gave up: let the gathers already in flight land before the CTA retires
+      for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
+        mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
+    }
+    __syncwarp();
   } else {
     // ---------------------------------------------------- softmax + read-out of O
     const int x = (warp - kSoftmaxWarp0) >> 2;     // 0: M tile A, 1: M tile B
@@ -923,7 +940,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const long long first = (long long)(w.ctx_begin + i) * kTileN;
             if (first + kTileN > w.Lj) limit = (int)(w.Lj - first);
           } else {
-            limit = min(t_row, p.Tq - 1) - (w.own_begin + i - w.n_ctx) * kTileN + 1;   // <= 0: all hidden
+            limit = p.To - p.Tq + min(t_row, p.Tq - 1) - (w.own_begin + i - w.n_ctx) * kTileN + 1;   // <= 0: all hidden
           }
           if (__any_sync(0xffffffffu, limit < kTileN)) {
 #pragma unroll
@@ -1002,8 +1019,8 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           unsigned char* stg = base_ptr + SM::kOffStage + (warp - kSoftmaxWarp0) * SM::kStageBytes;
           const int sub = lane >> 3, ch = lane & 7;            // read-back: row 4 j + sub, chunk ch
           const int m0 = mt * kTileM + quarter * 32;
-          if constexpr (MODE != kModeCache) {
-            // (no staging area in the shared-memory plan of the variants with loader warps: one row per thread)
+          if constexpr (FUSED) {
+            // (no staging area in the fused variant's shared-memory plan: one row per thread)
             const int hq = w.g * p.G + m % p.G;
             __nv_bfloat16* dst = p.out + (((bpj * p.Tq + t_row) * p.Hq) + hq) * (long long)D;
 #pragma unroll
@@ -1203,37 +1220,10 @@ __global__ void __launch_bounds__(64) wait_timeout_selftest_kernel(int32_t* stat
 }
 
 // ----------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
 // bf16 tensor, innermost dim contiguous, 128-byte swizzle, zero fill outside the bounds
 bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
               const uint32_t* box) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t gd[5], gs[4];
-  cuuint32_t bx[5], es[5];
-  for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
-  for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return ads_make_bf16_map(m, base, rank, dims, strides_bytes, box);
 }
 
 // Optional timing of the main kernel alone (adapshot_profile): two events around its launch.
@@ -1247,6 +1237,12 @@ struct AttnPlan {
   long long tab_rows;
 };
 
+// Own tokens beyond the query rows, and a per-query shot count on the device (decode calls).
+struct AttnExtra {
+  int To = 0;                        // 0: as many own tokens as query rows
+  const int32_t* nshots_dev = nullptr;
+};
+
 // What the fused variant reads instead of an assembled cache.
 struct FusedSrc {
   const adapshot_pool_t* pool;
@@ -1257,7 +1253,8 @@ struct FusedSrc {
 // The gang (CTAs that walk the same K/V tiles, one M pair each per round) is the number of
 // M pairs when that is at most kMaxGang, else the M pairs are dealt out in rounds.
 AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, long long fused_ctx_cap = 0,
-                   bool with_table = true) {
+                   bool with_table = true, int To = 0) {
+  if (To < Tq) To = Tq;
   AttnPlan pl;
   const int G = model->n_q_heads / model->n_kv_heads;
   const int D = model->head_dim;
@@ -1268,7 +1265,7 @@ AttnPlan make_plan(const adapshot_model_t* model, int B, int P, int Tq, int nl, 
   const size_t slots = (size_t)2 * kMaxCtas * pl.n_mp;     // two cut pieces per gang at most
   size_t off = 0;
   pl.off_qrot = off;  off += ads_round_up((size_t)B * nl * P * Tq * model->n_q_heads * D * 2, 256);
-  pl.off_kqrot = off; off += ads_round_up((size_t)B * nl * P * Tq * model->n_kv_heads * D * 2, 256);
+  pl.off_kqrot = off; off += ads_round_up((size_t)B * nl * P * To * model->n_kv_heads * D * 2, 256);
   pl.off_sched = off; off += ads_round_up(sizeof(Sched), 256);
   pl.off_opart = off; off += ads_round_up(slots * 2 * kTileM * D * 4, 256);
   pl.off_ml = off;    off += ads_round_up(slots * 2 * kTileM * 2 * 4, 256);
@@ -1294,7 +1291,8 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
                 const int64_t* ctx_off, int B, int k, const int32_t* probe_nshots, int P, const void* q,
                 const void* kq, const void* vq, int Tq, int nl, void* out, float* lse, const AttnPlan& pl,
                 void* ws, int32_t* status, cudaStream_t st, const FusedSrc* fused = nullptr,
-                int mode = kModeCache) {
+                int mode = kModeCache, AttnExtra extra = AttnExtra()) {
+  const int To = extra.To > Tq ? extra.To : Tq;
   const int Hq = model->n_q_heads, Hkv = model->n_kv_heads, G = Hq / Hkv;
   unsigned char* wsb = static_cast<unsigned char*>(ws);
   __nv_bfloat16* q_rot = reinterpret_cast<__nv_bfloat16*>(wsb + pl.off_qrot);
@@ -1326,11 +1324,23 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     if (mode == kModeCache && !make_map(&tm_vctx, v_ctx, 4, dims, str, box)) return ADAPSHOT_ECUDA;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)Tq, (uint64_t)B * nl * P};
-    const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, (uint64_t)Tq * Hkv * D * 2};
+    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, (uint64_t)To, (uint64_t)B * nl * P};
+    const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, (uint64_t)To * Hkv * D * 2};
     const uint32_t box[4] = {64, 1, (uint32_t)kTileN, 1};
     if (!make_map(&tm_kown, kq_rot, 4, dims, str, box)) return ADAPSHOT_ECUDA;
-    if (!make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    if (mode != kModeVPool && !make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+  }
+  if (mode == kModeVPool) {
+    // 2-D maps over all V rows (one row = the D values of one token and kv head) with one-row boxes:
+    // what the TMA row gather takes
+    const uint64_t str[1] = {(uint64_t)D * 2};
+    const uint32_t box[2] = {64, 1};
+    const uint64_t rows_pool = (uint64_t)model->n_layers * (uint64_t)fused->pool->pool_tokens * Hkv;
+    const uint64_t rows_own = (uint64_t)B * nl * P * To * Hkv;
+    if (rows_pool > 0x7fffffffull || rows_own > 0x7fffffffull) return ADAPSHOT_ESHAPE;   // row coordinates are int32
+    const uint64_t dims_pool[2] = {(uint64_t)D, rows_pool}, dims_own[2] = {(uint64_t)D, rows_own};
+    if (!make_map(&tm_vctx, fused->pool->v, 2, dims_pool, str, box)) return ADAPSHOT_ECUDA;
+    if (!make_map(&tm_vown, vq, 2, dims_own, str, box)) return ADAPSHOT_ECUDA;
   }
 
   // ---- fused variant: row map and rotary table
@@ -1359,10 +1369,11 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   pp.q_rot = q_rot; pp.kq_rot = kq_rot; pp.ctx_off = reinterpret_cast<const long long*>(ctx_off);
   pp.sched = sched; pp.ctx_cap = ctx_cap;
   pp.B = B; pp.k = k; pp.P = P; pp.Tq = Tq; pp.Hq = Hq; pp.Hkv = Hkv; pp.nl = nl; pp.n_gangs = n_gangs;
+  pp.To = To; pp.nshots_dev = extra.nshots_dev; pp.status = status;
   pp.rope_base = model->rope_base;
   for (int i = 0; i < D / 2; ++i) pp.theta[i] = pow(model->rope_base, -2.0 * (double)i / (double)D);
   for (int i = 0; i < kMaxProbes; ++i) pp.nshots[i] = i < P ? probe_nshots[i] : 0;
-  const long long n_tok = (long long)B * nl * P * Tq;
+  const long long n_tok = (long long)B * nl * P * To;
   attn_prep_kernel<D><<<(unsigned)((n_tok * kPrepParts + 7) / 8) + 1, 256, 0, st>>>(pp);   // + the schedule block
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
@@ -1370,7 +1381,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   AttnParams ap = {};
   ap.sched = sched; ap.o_part = o_part; ap.ml_part = ml_part;
   ap.out = static_cast<__nv_bfloat16*>(out); ap.lse = lse; ap.status = status;
-  ap.B = B; ap.P = P; ap.Tq = Tq; ap.Hq = Hq; ap.Hkv = Hkv; ap.G = G; ap.nl = nl;
+  ap.B = B; ap.P = P; ap.Tq = Tq; ap.Hq = Hq; ap.Hkv = Hkv; ap.G = G; ap.nl = nl; ap.To = To;
   ap.n_mt = pl.n_mt; ap.n_mp = pl.n_mp; ap.gang = pl.gang; ap.n_gangs = n_gangs;
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
@@ -1395,7 +1406,7 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
           tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
     } else {
       if (ads_set_max_smem(attn_main_kernel<D, kModeVPool>, smem, attr_done[2]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
-      attn_main_kernel<D, kModeVPool><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
+      attn_main_kernel<D, kModeVPool><<<(unsigned)(n_gangs * pl.gang), kVPoolThreads, smem, st>>>(
           tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
     }
   }
@@ -1551,6 +1562,117 @@ extern "C" int adapshot_query_attn_vpool(const adapshot_model_t* model, const ad
                             lse, pl, ws, status, st, &src, kModeVPool);
   return launch_attn<64>(model, k_ctx, nullptr, ctx_cap, ctx_off, B, k, probe_nshots, P, q, kq, vq, Tq, nl, out, lse,
                          pl, ws, status, st, &src, kModeVPool);
+}
+
+// ---------------------------------------------------------------- literal tree layout
+namespace {
+// Position ids of the probe tokens of the interleaved sequence: token t of probe j of query b sits
+// at L_j + t (the shots keep the positions 0 .. L-1 of their plain concatenation).
+struct TreePosArgs { int n[kMaxProbes]; };
+__global__ void tree_positions_kernel(const long long* __restrict__ ctx_off, int B, int k, int P, int Tq,
+                                           const TreePosArgs a, long long* __restrict__ pos) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)B * P * Tq) return;
+  const int t = (int)(i % Tq), j = (int)((i / Tq) % P), b = (int)(i / ((long long)Tq * P));
+  pos[i] = ctx_off[(long long)b * (k + 1) + a.n[j]] + t;
+}
+}  // namespace
+
+extern "C" int adapshot_tree_layout(const int32_t* seg_kind, const int32_t* seg_len, int32_t n_seg, int32_t k,
+                                    int32_t* probe_nshots, int32_t* P_out, int32_t* Tq_out) {
+  if (seg_kind == nullptr || seg_len == nullptr || probe_nshots == nullptr || P_out == nullptr || Tq_out == nullptr ||
+      n_seg <= 0)
+    return ADAPSHOT_EINVAL;
+  int shots = 0, P = 0, Tq = 0;
+  bool shots_since_probe = false;
+  for (int i = 0; i < n_seg; ++i) {
+    if (seg_len[i] <= 0) return ADAPSHOT_ESHAPE;
+    if (seg_kind[i] == ADAPSHOT_SEG_SHOTS) {
+      shots += seg_len[i];
+      if (shots > k) return ADAPSHOT_ESHAPE;
+      shots_since_probe = true;
+    } else if (seg_kind[i] == ADAPSHOT_SEG_PROBE) {
+      // every probe follows at least one new shot (nested counts are strictly ascending) and all
+      // probes have the same number of tokens
+      if (!shots_since_probe || P >= kMaxProbes) return ADAPSHOT_ESHAPE;
+      if (P == 0) Tq = seg_len[i];
+      else if (seg_len[i] != Tq) return ADAPSHOT_ESHAPE;
+      probe_nshots[P++] = shots;
+      shots_since_probe = false;
+    } else {
+      return ADAPSHOT_EINVAL;
+    }
+  }
+  if (P == 0 || shots_since_probe) return ADAPSHOT_ESHAPE;      // the sequence ends with a probe
+  *P_out = P;
+  *Tq_out = Tq;
+  return ADAPSHOT_OK;
+}
+
+extern "C" int adapshot_tree_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx,
+                                  int64_t ctx_cap, const int64_t* ctx_off, int32_t B, int32_t k,
+                                  const int32_t* seg_kind, const int32_t* seg_len, int32_t n_seg,
+                                  const void* q_seq, const void* kq_seq, const void* vq_seq,
+                                  int32_t layer_begin, int32_t layer_end, void* out_seq, float* lse,
+                                  int64_t* pos_seq, uint32_t flags, void* ws, size_t ws_bytes, int32_t* status,
+                                  void* stream) {
+  int32_t nshots[kMaxProbes], P = 0, Tq = 0;
+  if (model == nullptr || ctx_off == nullptr) return ADAPSHOT_EINVAL;
+  const int rc = adapshot_tree_layout(seg_kind, seg_len, n_seg, k, nshots, &P, &Tq);
+  if (rc != ADAPSHOT_OK) return rc;
+  // the probe tokens of the sequence, in sequence order, are [P][T_q]: the per-probe call's layout
+  const int rc2 = adapshot_query_attn(model, k_ctx, v_ctx, ctx_cap, ctx_off, B, k, nshots, P, q_seq, kq_seq, vq_seq,
+                                      Tq, layer_begin, layer_end, out_seq, lse, flags, ws, ws_bytes, status, stream);
+  if (rc2 != ADAPSHOT_OK || pos_seq == nullptr) return rc2;
+  if ((uintptr_t)pos_seq & 7u) return ADAPSHOT_EALIGN;
+  TreePosArgs a;
+  for (int i = 0; i < kMaxProbes; ++i) a.n[i] = i < P ? nshots[i] : 0;
+  const long long n = (long long)B * P * Tq;
+  tree_positions_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<const long long*>(ctx_off), B, k, P, Tq, a, reinterpret_cast<long long*>(pos_seq));
+  return ads_launch_status();
+}
+
+// ------------------------------------------------------------------------ decode step
+extern "C" size_t adapshot_decode_workspace_bytes(const adapshot_model_t* model, int32_t B, int32_t T_new,
+                                                  int32_t T_own, int32_t n_layers_in_call) {
+  if (model == nullptr || !attn_shape_ok(model) || B <= 0 || T_new <= 0 || T_own < T_new || n_layers_in_call <= 0)
+    return 0;
+  return make_plan(model, B, 1, T_new, n_layers_in_call, 0, true, T_own).total;
+}
+
+extern "C" int adapshot_decode_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_ctx,
+                                    int64_t ctx_cap, const int64_t* ctx_off, int32_t B, int32_t k,
+                                    const int32_t* n_shots, const void* q_new, const void* k_own,
+                                    const void* v_own, int32_t T_new, int32_t T_own, int32_t layer_begin,
+                                    int32_t layer_end, void* out, float* lse, uint32_t flags, void* ws,
+                                    size_t ws_bytes, int32_t* status, void* stream) {
+  if (model == nullptr || k_ctx == nullptr || v_ctx == nullptr || ctx_off == nullptr || n_shots == nullptr ||
+      q_new == nullptr || k_own == nullptr || v_own == nullptr || out == nullptr || ws == nullptr)
+    return ADAPSHOT_EINVAL;
+  if (B <= 0 || k <= 0 || T_new <= 0 || ctx_cap <= 0 || flags != 0) return ADAPSHOT_EINVAL;
+  if (T_own < T_new) return ADAPSHOT_ESHAPE;
+  if (model->dtype != ADAPSHOT_BF16) return ADAPSHOT_EUNSUPPORTED;
+  if (!attn_shape_ok(model)) return ADAPSHOT_ESHAPE;
+  if (layer_begin < 0 || layer_end <= layer_begin || layer_end > model->n_layers) return ADAPSHOT_ESHAPE;
+  if (B > kMaxPairs) return ADAPSHOT_ESHAPE;
+  if (!ads_aligned16(k_ctx) || !ads_aligned16(v_ctx) || !ads_aligned16(q_new) || !ads_aligned16(k_own) ||
+      !ads_aligned16(v_own) || !ads_aligned16(out) || ((uintptr_t)ws & 255u) || ((uintptr_t)n_shots & 3u))
+    return ADAPSHOT_EALIGN;
+  if (ctx_cap > (1ll << 31) - 256) return ADAPSHOT_ESHAPE;
+  const int nl = layer_end - layer_begin;
+  const AttnPlan pl = make_plan(model, B, 1, T_new, nl, 0, true, T_own);
+  if (ws_bytes < pl.total) return ADAPSHOT_ECAPACITY;
+  AttnExtra extra;
+  extra.To = T_own;
+  extra.nshots_dev = n_shots;
+  const int32_t one = 1;      // (placeholder for the host list: the per-query device counts are used)
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (model->head_dim == 128)
+    return launch_attn<128>(model, k_ctx, v_ctx, ctx_cap, ctx_off, B, k, &one, 1, q_new, k_own, v_own, T_new, nl, out,
+                            lse, pl, ws, status, st, nullptr, kModeCache, extra);
+  return launch_attn<64>(model, k_ctx, v_ctx, ctx_cap, ctx_off, B, k, &one, 1, q_new, k_own, v_own, T_new, nl, out,
+                         lse, pl, ws, status, st, nullptr, kModeCache, extra);
 }
 
 extern "C" int adapshot_profile(int enable) {

@@ -62,6 +62,26 @@ __device__ __forceinline__ void ads_set_status(int32_t* status, int32_t code) {
   if (status != nullptr) atomicCAS(status, 0, code);
 }
 
+// Order-preserving map of an fp64 score to an unsigned key; larger score -> SMALLER key so that an
+// ascending order on (key, id) lists the most relevant shot first and equal scores by ascending id.
+__device__ __forceinline__ unsigned long long ads_desc_key(double s) {
+  unsigned long long u = (unsigned long long)__double_as_longlong(s);
+  u = (u >> 63) ? ~u : (u | 0x8000000000000000ull);   // ascending in s
+  return ~u;
+}
+__device__ __forceinline__ double ads_key_score(unsigned long long k) {
+  unsigned long long u = ~k;
+  u = (u >> 63) ? (u & 0x7fffffffffffffffull) : ~u;
+  return __longlong_as_double((long long)u);
+}
+
+// Top k of N candidates per query from their sort keys (select.cu): keys [B][N] as ads_desc_key
+// writes them, ids [B][N] = 0..N-1 (read only when N needs the chunked sort), cand = scratch of
+// ads_topk_scratch_bytes(N, B, k) bytes.  Enqueues on st; returns an ADAPSHOT_* code.
+size_t ads_topk_scratch_bytes(int N, int B, int k);
+int ads_topk_from_keys(const unsigned long long* keys, const int* ids, int N, int B, int k, void* cand,
+                       int32_t* sel_idx, float* sel_score, cudaStream_t st);
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

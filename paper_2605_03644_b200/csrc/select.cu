@@ -13,19 +13,8 @@ namespace {
 constexpr int kSortCap = 8192;      // candidates one CTA sorts in shared memory
 constexpr int kSortThreads = 1024;
 
-// Order-preserving map of an fp64 score to an unsigned key; larger score -> SMALLER
-// key so that an ascending sort on (key, id) lists the most relevant shot first and
-// equal scores by ascending id.
-__device__ __forceinline__ unsigned long long desc_key(double s) {
-  unsigned long long u = (unsigned long long)__double_as_longlong(s);
-  u = (u >> 63) ? ~u : (u | 0x8000000000000000ull);   // ascending in s
-  return ~u;
-}
-__device__ __forceinline__ double key_score(unsigned long long k) {
-  unsigned long long u = ~k;
-  u = (u >> 63) ? (u & 0x7fffffffffffffffull) : ~u;
-  return __longlong_as_double((long long)u);
-}
+__device__ __forceinline__ unsigned long long desc_key(double s) { return ads_desc_key(s); }
+__device__ __forceinline__ double key_score(unsigned long long k) { return ads_key_score(k); }
 
 // One warp per pool row i: dots[b][i] = <q_b, e_i> for all b, enorm[i] = |e_i|.  With
 // keys_out set (pools that the rank kernel handles) the warp also forms |q_b| from the values
@@ -230,6 +219,55 @@ size_t sel_cand_entries(int n_shots, int k) {
 }
 
 }  // namespace
+
+size_t ads_topk_scratch_bytes(int N, int B, int k) {
+  const size_t cand = sel_cand_entries(N, k);
+  return 2 * (ads_round_up((size_t)B * cand * 8, 256) + ads_round_up((size_t)B * cand * 4, 256));
+}
+
+int ads_topk_from_keys(const unsigned long long* keys, const int* ids, int N, int B, int k, void* cand_ws,
+                       int32_t* sel_idx, float* sel_score, cudaStream_t st) {
+  if (N > kSortCap && k > kSortCap / 2) return ADAPSHOT_EUNSUPPORTED;
+  if (N <= kRankMaxN) {
+    dim3 grid((N + kRankCand - 1) / kRankCand, B);
+    rank_topk_kernel<<<grid, kRankThreads, 0, st>>>(keys, N, k, sel_idx, sel_score);
+    return ads_launch_status();
+  }
+  const size_t smem = (size_t)kSortCap * (8 + 4);
+  static bool attr_set[kAdsMaxDevices] = {false};
+  if (ads_set_max_smem(topk_sort_kernel, (int)smem, attr_set) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+  const size_t cand = sel_cand_entries(N, k);
+  unsigned char* p = static_cast<unsigned char*>(cand_ws);
+  unsigned long long* ckey[2];
+  int* cid[2];
+  for (int i = 0; i < 2; ++i) {
+    ckey[i] = reinterpret_cast<unsigned long long*>(p);
+    p += ads_round_up((size_t)B * cand * 8, 256);
+    cid[i] = reinterpret_cast<int*>(p);
+    p += ads_round_up((size_t)B * cand * 4, 256);
+  }
+  int n_in = N, in_stride = N, round = 0;
+  const unsigned long long* in_key = keys;
+  const int* in_id = ids;
+  while (true) {
+    const int chunks = (n_in + kSortCap - 1) / kSortCap;
+    const bool last = chunks == 1;
+    dim3 grid(chunks, B);
+    const int out_stride = chunks * k;
+    topk_sort_kernel<<<grid, kSortThreads, smem, st>>>(
+        nullptr, nullptr, nullptr, 0, in_key, in_id, n_in, in_stride, k, ckey[round & 1], cid[round & 1], out_stride,
+        last ? sel_idx : nullptr, last ? sel_score : nullptr);
+    if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
+    if (last) break;
+    in_key = ckey[round & 1];
+    in_id = cid[round & 1];
+    const int last_n = n_in - (chunks - 1) * kSortCap;
+    n_in = (chunks - 1) * k + (last_n < k ? last_n : k);
+    in_stride = out_stride;
+    ++round;
+  }
+  return ADAPSHOT_OK;
+}
 
 extern "C" size_t adapshot_select_workspace_bytes(int32_t n_shots, int32_t B, int32_t k) {
   if (n_shots <= 0 || B <= 0 || k <= 0) return 0;
