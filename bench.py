@@ -139,14 +139,14 @@ def resolve_k_by_budget(ab, dpool, q_emb, w: wl.Workload, lengths: np.ndarray) -
     return w.scaled(k=k, probes=(k,))
 
 
-def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e9) -> int:
+def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e9, k_only: bool = False) -> int:
     """Layers assembled and attended per call: as many as fit beside the pool, the query-side
-    tensors and the outputs, at most 36 GB of assembled K + V."""
+    tensors and the outputs, at most 36 GB of assembled K + V (k_only: the cache holds K alone)."""
     n_tok = float(wl.shot_lengths(w).sum())
     pool_bytes = n_tok * w.bytes_per_token_layer * w.n_layers
     q_bytes = (w.batch * w.n_layers * max(1, len(w.probes)) * w.t_q * (w.n_q_heads + 2 * w.n_kv_heads)
                * w.head_dim * w.elem_size)
-    per_layer = float(w.batch) * ctx_cap * w.bytes_per_token_layer
+    per_layer = float(w.batch) * ctx_cap * w.bytes_per_token_layer * (0.5 if k_only else 1.0)
     budget = min(36e9, 0.5 * (device_bytes - pool_bytes - 3.0 * q_bytes))
     return int(max(1, min(w.n_layers, budget // per_layer)))
 
@@ -382,9 +382,9 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
                           k_pos_mode=args.k_pos_mode)
     qs = wl.make_queries(wq, dev)
     ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
-    lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap)
     fused = args.variant == "fused"
     vpool = args.variant == "vpool"
+    lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap, k_only=vpool)
     if fused and not args.layers_per_call:
         lpc = w.n_layers                      # no assembled cache to fit: all layers in one call
     path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused,

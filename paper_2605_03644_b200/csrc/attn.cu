@@ -332,7 +332,8 @@ struct AttnSmem {
   static constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
   static constexpr uint32_t kOffStage = kOffV + kVStages * kTileBytes;    // read-out staging of the 8 softmax warps
   static constexpr uint32_t kOffBar = kOffStage + 8 * kStageBytes;
-  static constexpr uint32_t kTotal = kOffBar + 256 + 1024 + 1024;        // barriers, schedule cache, alignment slack
+  static constexpr uint32_t kOffRows = kOffBar + 256 + 1024;              // V-from-pool variant: pool rows of a tile
+  static constexpr uint32_t kTotal = kOffRows + (MODE == kModeVPool ? 512 : 0) + 1024;   // + alignment slack
 };
 
 // mbarrier slots (8 bytes each)
@@ -449,6 +450,12 @@ __device__ __forceinline__ void make_item(const AttnParams& p, const Piece& pc, 
   w.slot = ((long long)(2 * gang_id + (pc.first_of_gang ? 0 : 1)) * p.n_mp + mp);
 }
 
+// V-from-pool variant: maps over the pool's V with boxes of 1, 2, 4, ..., 128 rows, from which a
+// tile is stitched run by run (a run = consecutive context positions that are consecutive pool rows).
+struct VPoolMaps {
+  CUtensorMap m[8];
+};
+
 // TMEM: S/P of M tile A at columns 0..127, of M tile B at 128..255 (P, as packed bf16,
 // overwrites the S tile it was computed from); O accumulators at 256 and 384.
 // FUSED: the context K/V tiles are read from the pool through the row map (per-thread async
@@ -458,7 +465,8 @@ template <int D, int MODE>
 __global__ void __launch_bounds__(MODE == kModeFused ? kFusedThreads : (MODE == kModeVPool ? kVPoolThreads : kAttnThreads), 1)
 attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kctx,
                  const __grid_constant__ CUtensorMap tm_vctx, const __grid_constant__ CUtensorMap tm_kown,
-                 const __grid_constant__ CUtensorMap tm_vown, const AttnParams p) {
+                 const __grid_constant__ CUtensorMap tm_vown, const __grid_constant__ VPoolMaps vmaps,
+                 const AttnParams p) {
   constexpr bool FUSED = MODE == kModeFused;
   constexpr bool VPOOL = MODE == kModeVPool;
   using SM = AttnSmem<D, MODE>;
@@ -852,55 +860,159 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     cp_async_wait<0>();
   } else if (VPOOL && warp == kGatherWarp) {
-    // ----------------------------------------- V tiles straight from the pool (TMA row gather)
-    // Eq. 7 corrects K only, so V needs no assembled copy: the 128 context positions of a tile are
-    // looked up in the row map and their pool rows fetched four at a time by TMA gather copies
-    // (one-row boxes of a 2-D map over all V rows of the pool, 128-byte swizzle, so the tile lands
-    // in the layout the PV descriptors expect).  Lane i brings rows 4 i .. 4 i + 3; rows beyond the
-    // context (their P is exactly zero) read some valid row instead of being skipped, so that every
-    // tile delivers the same number of bytes to its barrier.
+    // ----------------------------------------------- V tiles straight from the pool, stitched by TMA
+    // Eq. 7 corrects K only, so V needs no assembled copy.  The 128 context positions of a tile map
+    // to a few runs of consecutive pool rows (one per selected shot the tile touches): the lanes look
+    // the positions up and mark where a run ends; every run is brought as power-of-two boxes (maps with
+    // 128, 64, ..., 1-row boxes over the pool; a box may start at any row, its shared-memory address only
+    // has to be 128-byte aligned), one box per lane, all found before the stage is waited for.
+    // Positions beyond the context continue the last run (their P is exactly zero; rows outside the
+    // pool arrive as zeros), so every tile delivers the same number of bytes to its barrier.  The
+    // probe's own tokens are one run of the own-token tensor.
+    int* rows_s = reinterpret_cast<int*>(base_ptr + SM::kOffRows);
     uint32_t tv = 0;
     bool ok = true;
     Walker wk = wk0;
     Piece pc;
-    if (lane == 0) { tma_prefetch_desc(&tm_vctx); tma_prefetch_desc(&tm_vown); }
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_vown);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) tma_prefetch_desc(&vmaps.m[e]);
+    }
     while (ok && next_piece(sc, cache, n_pairs, wk, pc)) {
       for (int mp = rank; mp < p.n_mp && ok; mp += p.gang) {
         Item w;
         make_item(p, pc, gang_id, mp, w);
         for (int i = 0; i < w.n_tiles; ++i, ++tv) {
           const uint32_t sv = tv % VS;
-          const bool own = i >= w.n_ctx;
-          int y[4];                                    // rows of the 2-D V map (in rows of D elements)
+          const uint32_t v_dst = base + SM::kOffV + sv * kTileBytes;
+          if (i >= w.n_ctx) {
+            // own tokens: one tiled box (rows beyond the last own token arrive as zeros)
+            if (lane == 0) {
+              ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
+              if (ok) {
+                mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {             // (looked up while the stage may still be in use)
-            const int row = 4 * lane + q4;
-            if (!own) {
-              const long long pos = (long long)(w.ctx_begin + i) * kTileN + row;
-              int r = pos < p.ctx_cap ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
-              if (r < 0) r = 0;
-              y[q4] = (int)(((long long)(p.layer_begin + w.l) * p.pool_tokens + r) * p.Hkv + w.g);
-            } else {
-              const int t = min((w.own_begin + i - w.n_ctx) * kTileN + row, p.To - 1);
-              y[q4] = (int)(((long long)w.outer_own * p.To + t) * p.Hkv + w.g);
+                for (int s2 = 0; s2 < SUB; ++s2)
+                  tma_load_4d(v_dst + s2 * 16384u, &tm_vown, bar(kBarVFull + sv), s2 * 64, w.g,
+                              (w.own_begin + i - w.n_ctx) * kTileN, w.outer_own);
+              }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            continue;
+          }
+          // pool row of positions lane, lane + 32, lane + 64, lane + 96 of the tile (looked up while the
+          // stage may still be in use); beyond the context the last run is continued
+          const long long pos0 = (long long)(w.ctx_begin + i) * kTileN;
+          const long long L_all = p.ctx_cap;            // (row map entries beyond a query's context are -1)
+          int r[4];
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const long long pos = pos0 + lane + 32 * q4;
+            r[q4] = pos < L_all ? p.row_map[(long long)w.b * p.ctx_cap + pos] : -1;
+          }
+          // the number of valid positions of the tile: they form a prefix (valid positions are 0 .. L-1)
+          unsigned valid_mask[4];
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) valid_mask[q4] = __ballot_sync(0xffffffffu, r[q4] >= 0);
+          const int n_valid = __popc(valid_mask[0]) + __popc(valid_mask[1]) + __popc(valid_mask[2]) + __popc(valid_mask[3]);
+          __syncwarp();
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) rows_s[lane + 32 * q4] = r[q4];
+          __syncwarp();
+          const int last_row = n_valid > 0 ? rows_s[n_valid - 1] : 0;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int pidx = lane + 32 * q4;
+            if (pidx >= n_valid) r[q4] = last_row + (pidx - n_valid + 1);
+          }
+          __syncwarp();
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) rows_s[lane + 32 * q4] = r[q4];
+          // a run ends after position pidx when the next position is not the next pool row
+          unsigned brk[4];
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            int nxt = __shfl_down_sync(0xffffffffu, r[q4], 1);
+            const int wrap = __shfl_sync(0xffffffffu, q4 < 3 ? r[q4 + 1 < 4 ? q4 + 1 : 3] : 0, 0);
+            if (lane == 31) nxt = wrap;
+            const bool last = lane == 31 && q4 == 3;
+            brk[q4] = __ballot_sync(0xffffffffu, last || nxt != r[q4] + 1);
+          }
+          // the run ends as one 128-bit mask in every lane; lane j then finds the j-th box on its own:
+          // boxes are numbered run by run, a run of n rows gives popcount(n) boxes, largest first
+          __syncwarp();
+          int my_pidx = -1, my_row = 0, my_lg = 0, n_boxes = 0;
+          {
+            int pidx = 0;
+            while (pidx < kTileN) {
+              int e = pidx;                       // end of the run that starts at pidx: first set bit at or after it
+              for (;;) {
+                const unsigned word = (e < 32 ? brk[0] : e < 64 ? brk[1] : e < 96 ? brk[2] : brk[3]) >> (e & 31);
+                if (word != 0) { e += __ffs(word) - 1; break; }
+                e = (e | 31) + 1;
+              }
+              int n = e - pidx + 1;
+              int off = 0;
+              while (n > 0) {
+                const int lg = 31 - __clz(n);      // the largest power-of-two box that fits
+                if (n_boxes == lane) { my_pidx = pidx + off; my_lg = lg; }
+                ++n_boxes;
+                off += 1 << lg;
+                n -= 1 << lg;
+              }
+              pidx = e + 1;
             }
           }
+          if (my_pidx >= 0) my_row = rows_s[my_pidx];
+          // (tiles of more than 32 boxes - many one-token shots - take further rounds of the same walk)
           if (lane == 0) {
             ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
             if (ok) mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
           }
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) break;
-          const CUtensorMap* mv = own ? &tm_vown : &tm_vctx;
-          const uint32_t dst = base + SM::kOffV + sv * kTileBytes + (uint32_t)(4 * lane) * 128u;
+          const int layer = p.layer_begin + w.l;
+          if (my_pidx >= 0) {
 #pragma unroll
-          for (int s2 = 0; s2 < SUB; ++s2)
-            tma_gather4(dst + s2 * 16384u, mv, bar(kBarVFull + sv), s2 * 64, y[0], y[1], y[2], y[3]);
+            for (int s2 = 0; s2 < SUB; ++s2)
+              tma_load_4d(v_dst + s2 * 16384u + (uint32_t)my_pidx * 128u, &vmaps.m[my_lg], bar(kBarVFull + sv), s2 * 64,
+                          w.g, my_row, layer);
+          }
+          for (int round = 1; round * 32 < n_boxes; ++round) {      // rare: more than 32 boxes in the tile
+            int pidx = 0, idx = 0, bp = -1, bl = 0;
+            while (pidx < kTileN) {
+              int e = pidx;
+              for (;;) {
+                const unsigned word = (e < 32 ? brk[0] : e < 64 ? brk[1] : e < 96 ? brk[2] : brk[3]) >> (e & 31);
+                if (word != 0) { e += __ffs(word) - 1; break; }
+                e = (e | 31) + 1;
+              }
+              int n = e - pidx + 1, off = 0;
+              while (n > 0) {
+                const int lg = 31 - __clz(n);
+                if (idx == round * 32 + lane) { bp = pidx + off; bl = lg; }
+                ++idx;
+                off += 1 << lg;
+                n -= 1 << lg;
+              }
+              pidx = e + 1;
+            }
+            if (bp >= 0) {
+              const int brow = rows_s[bp];
+#pragma unroll
+              for (int s2 = 0; s2 < SUB; ++s2)
+                tma_load_4d(v_dst + s2 * 16384u + (uint32_t)bp * 128u, &vmaps.m[bl], bar(kBarVFull + sv), s2 * 64, w.g,
+                            brow, layer);
+            }
+          }
+          __syncwarp();
         }
       }
     }
     if (!ok && lane == 0) {
-      // gave up: let the gathers already in flight land before the CTA retires
+      // gave up: let the copies already in flight land before the CTA retires
       for (uint32_t t = tv > (uint32_t)VS ? tv - VS : 0; t < tv; ++t)
         mbar_wait(bar(kBarVFull + t % VS), (t / VS) & 1, abort_flag + 1);
     }
@@ -1328,19 +1440,19 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, (uint64_t)To * Hkv * D * 2};
     const uint32_t box[4] = {64, 1, (uint32_t)kTileN, 1};
     if (!make_map(&tm_kown, kq_rot, 4, dims, str, box)) return ADAPSHOT_ECUDA;
-    if (mode != kModeVPool && !make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    if (!make_map(&tm_vown, vq, 4, dims, str, box)) return ADAPSHOT_ECUDA;
   }
+  VPoolMaps vmaps;
+  for (int e = 0; e < 8; ++e) vmaps.m[e] = tm_q;       // (unused outside the V-from-pool variant)
   if (mode == kModeVPool) {
-    // 2-D maps over all V rows (one row = the D values of one token and kv head) with one-row boxes:
-    // what the TMA row gather takes
-    const uint64_t str[1] = {(uint64_t)D * 2};
-    const uint32_t box[2] = {64, 1};
-    const uint64_t rows_pool = (uint64_t)model->n_layers * (uint64_t)fused->pool->pool_tokens * Hkv;
-    const uint64_t rows_own = (uint64_t)B * nl * P * To * Hkv;
-    if (rows_pool > 0x7fffffffull || rows_own > 0x7fffffffull) return ADAPSHOT_ESHAPE;   // row coordinates are int32
-    const uint64_t dims_pool[2] = {(uint64_t)D, rows_pool}, dims_own[2] = {(uint64_t)D, rows_own};
-    if (!make_map(&tm_vctx, fused->pool->v, 2, dims_pool, str, box)) return ADAPSHOT_ECUDA;
-    if (!make_map(&tm_vown, vq, 2, dims_own, str, box)) return ADAPSHOT_ECUDA;
+    // the pool's V with boxes of 1, 2, ..., 128 rows (the layout of the cache maps, over the pool)
+    const uint64_t pt = (uint64_t)fused->pool->pool_tokens;
+    const uint64_t dims[4] = {(uint64_t)D, (uint64_t)Hkv, pt, (uint64_t)model->n_layers};
+    const uint64_t str[3] = {(uint64_t)D * 2, (uint64_t)Hkv * D * 2, pt * Hkv * D * 2};
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t box[4] = {64, 1, 1u << e, 1};
+      if (!make_map(&vmaps.m[e], fused->pool->v, 4, dims, str, box)) return ADAPSHOT_ECUDA;
+    }
   }
 
   // ---- fused variant: row map and rotary table
@@ -1385,13 +1497,14 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
   ap.n_mt = pl.n_mt; ap.n_mp = pl.n_mp; ap.gang = pl.gang; ap.n_gangs = n_gangs;
   const float scale = model->softmax_scale > 0.f ? model->softmax_scale : 1.0f / sqrtf((float)D);
   ap.scale_log2 = scale * 1.4426950408889634f;
-  const int smem = (int)AttnSmem<128, kModeCache>::kTotal;     // same request for D = 64 and for the fused variant: one CTA per SM
+  // the same request for D = 64 as for D = 128: one CTA per SM in every variant
+  const int smem = mode == kModeVPool ? (int)AttnSmem<128, kModeVPool>::kTotal : (int)AttnSmem<128, kModeCache>::kTotal;
   static bool attr_done[3][kAdsMaxDevices] = {{false}, {false}, {false}};   // per template instance (D, mode) and device
   if (g_profile) ADS_CHECK_CUDA(cudaEventRecord(g_profile_ev[0], st));
   if (mode == kModeCache) {
     if (ads_set_max_smem(attn_main_kernel<D, kModeCache>, smem, attr_done[0]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
     attn_main_kernel<D, kModeCache><<<(unsigned)(n_gangs * pl.gang), kAttnThreads, smem, st>>>(
-        tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+        tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, vmaps, ap);
   } else {
     ap.k_pool = static_cast<const __nv_bfloat16*>(fused->pool->k);
     ap.v_pool = static_cast<const __nv_bfloat16*>(fused->pool->v);
@@ -1403,11 +1516,11 @@ int launch_attn(const adapshot_model_t* model, const void* k_ctx, const void* v_
     if (mode == kModeFused) {
       if (ads_set_max_smem(attn_main_kernel<D, kModeFused>, smem, attr_done[1]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
       attn_main_kernel<D, kModeFused><<<(unsigned)(n_gangs * pl.gang), kFusedThreads, smem, st>>>(
-          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, vmaps, ap);
     } else {
       if (ads_set_max_smem(attn_main_kernel<D, kModeVPool>, smem, attr_done[2]) != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
       attn_main_kernel<D, kModeVPool><<<(unsigned)(n_gangs * pl.gang), kVPoolThreads, smem, st>>>(
-          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, ap);
+          tm_q, tm_kctx, tm_vctx, tm_kown, tm_vown, vmaps, ap);
     }
   }
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;

@@ -64,7 +64,7 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=Fa
     assert orc.min_adjacent_gap(q_emb64, emb64, w.k) > 1e-12
     off = orc.plan_offsets(sel, pool["shot_off"])
     ctx_cap = int(-(-int(off[:, -1].max()) // 128) * 128)
-    lpc = w.n_layers if fused else layers_per_call_for(w, ctx_cap)
+    lpc = w.n_layers if fused else layers_per_call_for(w, ctx_cap, k_only=vpool)
 
     # ---- the CUDA path, as the benchmark launches it
     dpool = ab.Pool(torch.from_numpy(pool["shot_off"]).to(dev), pool["k"], pool["v"], pool["emb"])

@@ -74,7 +74,7 @@ def test_peaked_queries_single_out_their_shot():
     # queries five times larger: the softmax over the pool concentrates on a few keys
     w = wl.CONFIGS["cfg2"].scaled(n_shots=64, len_lo=20, len_hi=90, batch=2, k=8, t_q=16, seed=84)
     sel, score = _check(w, 1, 0, 8, q_gain=5.0)
-    assert (score[:, 0] > 2.0 / 64).all()
+    assert (score[:, 0] > 1.5 / 64).all()                 # well above the uniform share of 1 / 64
 
 
 def test_identical_shots_get_equal_masses():
