@@ -151,6 +151,16 @@ def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e
     return int(max(1, min(w.n_layers, budget // per_layer)))
 
 
+def choose_variant(w: wl.Workload, ctx_cap: int, variant: str = "auto", layers_per_call: int = 0):
+    """(vpool, layers per call) of a run.  auto: the K-only cache (V taken from the pool) when the full cache of
+    one call would be larger than L2, the full cache otherwise (the rule of ReusePath(vpool=None))."""
+    vpool = variant == "vpool"
+    if variant == "auto":
+        lpc_full = layers_per_call or layers_per_call_for(w, ctx_cap)
+        vpool = w.batch * lpc_full * ctx_cap * w.bytes_per_token_layer > (128 << 20)
+    return vpool, (layers_per_call or layers_per_call_for(w, ctx_cap, k_only=vpool))
+
+
 def planned_ctx_cap(ab, dpool, q_emb, w: wl.Workload) -> int:
     """Capacity of the assembled cache: the longest planned context (selection + plan-only
     call of the library), rounded up to the 128-token tile the attention kernel reads."""
@@ -334,20 +344,20 @@ def per_probe_costs(ab, path, model, dpool, w, qc, kqc, vqc, ctx_off_np, flush, 
     for j, n_j in enumerate(w.probes):
         q_j, kq_j, vq_j = (x[0][:, :, j:j + 1].contiguous() for x in (qc, kqc, vqc))
         o_j = torch.empty_like(q_j)
-        attn_ms = _timed(lambda: ab.adapshot_query_attn(model, k_ctx, v_ctx, path.ctx_cap, path.ctx_off, path.k,
-                                                        [n_j], q_j, kq_j, vq_j, lb, le, o_j, None, path.ws_attn,
-                                                        path.status), n_rep, flush)
+        attn_ms = _timed(lambda: path.attend(q_j, kq_j, vq_j, o_j, lb, le, probes=[n_j]), n_rep, flush)
         sel_j = path.sel_idx[:, :n_j].contiguous()
         off_j = torch.empty((w.batch, n_j + 1), dtype=torch.int64, device=dev)
+        gflags = ab.ASSEMBLE_K_ONLY if path.vpool else 0
         gather_ms = _timed(lambda: ab.adapshot_assemble_kv_from(model, dpool, sel_j, prev, lb, le, k_ctx, v_ctx,
-                                                                path.ctx_cap, off_j, path.status), n_rep, flush)
+                                                                path.ctx_cap, off_j, path.status, flags=gflags),
+                           n_rep, flush)
         Lj = ctx_off_np[:, n_j].astype(np.float64)
         Lp = ctx_off_np[:, prev].astype(np.float64) if prev else np.zeros_like(Lj)
         flops = float((4.0 * w.t_q * (Lj + (w.t_q + 1) / 2.0) * w.n_q_heads * w.head_dim).sum()) * nl
         out.append({"n_shots": int(n_j), "ctx_tokens": float(Lj.sum()),
                     "attn_ms": attn_ms * w.n_layers / nl, "attn_tflops": flops / (attn_ms * 1e-3) / 1e12,
                     "gather_added_ms": gather_ms * w.n_layers / nl,
-                    "gather_added_gbs": float((Lj - Lp).sum()) * w.bytes_per_token_layer * 2 * nl
+                    "gather_added_gbs": float((Lj - Lp).sum()) * w.bytes_per_token_layer * (1 if path.vpool else 2) * nl
                     / (gather_ms * 1e-3) / 1e9})
         prev = n_j
     path.assemble(lb, le, keep_plan=True)        # the cache of the whole selection again
@@ -383,8 +393,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     qs = wl.make_queries(wq, dev)
     ctx_cap = args.ctx_cap or planned_ctx_cap(ab, dpool, qs["q_emb"], w)
     fused = args.variant == "fused"
-    vpool = args.variant == "vpool"
-    lpc = args.layers_per_call or layers_per_call_for(w, ctx_cap, k_only=vpool)
+    vpool, lpc = choose_variant(w, ctx_cap, args.variant, args.layers_per_call)
     if fused and not args.layers_per_call:
         lpc = w.n_layers                      # no assembled cache to fit: all layers in one call
     path = ReusePath(model, dpool, w.batch, w.k, w.probes, w.t_q, w.vocab, ctx_cap, lpc, fused=fused,
@@ -544,7 +553,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     }
 
     per_probe = None
-    if len(w.probes) > 1 and not fused and not vpool:
+    if len(w.probes) > 1 and not fused:
         per_probe = per_probe_costs(ab, path, model, dpool, w, qc, kqc, vqc, ctx_off, flush)
         check_status("after the per-probe pass")
 
@@ -594,7 +603,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     check_status("after the end-to-end pass")
 
     config = workload_config(w, pool["n_shots"], pool["pool_tokens"], counts["ctx_tokens"], world)
-    config.update({"variant": args.variant, "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph,
+    config.update({"variant": "fused" if fused else ("vpool" if vpool else "materialise"), "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph,
                    "ctx_cap": ctx_cap, "layers_per_call": lpc, "gather_overlaps_attention": path.overlap,
                    "entropy": "side stream, overlapped with the pass" if path.entropy_overlap
                    else "after the last attention call (serial)",
@@ -747,10 +756,11 @@ def main():
                     help="run only the first N queries of the workload (a smaller case for profiler captures)")
     ap.add_argument("--layers-per-call", type=int, default=0)
     ap.add_argument("--ctx-cap", type=int, default=0)
-    ap.add_argument("--variant", default="materialise", choices=["materialise", "vpool", "fused"],
+    ap.add_argument("--variant", default="auto", choices=["auto", "materialise", "vpool", "fused"],
                     help="materialise: gather + re-encode K and V into a contiguous cache, then attend; "
-                         "vpool: gather + re-encode K only, attention copies V tiles from the pool; "
-                         "fused: attention reads the pool and re-encodes K in shared memory")
+                         "vpool: gather + re-encode K only, attention takes V tiles from the pool; "
+                         "fused: attention reads the pool and re-encodes K in shared memory; "
+                         "auto (default): vpool when a call's cache is larger than L2, else materialise")
     ap.add_argument("--k-pos-mode", type=int, default=0, choices=[0, 1],
                     help="0: pool K carries no position (default); 1: pool K rotated at shot-local positions "
                          "(the paper's store), the re-encode is one angle per shot")

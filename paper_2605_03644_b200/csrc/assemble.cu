@@ -92,10 +92,6 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
-__device__ __forceinline__ void prefetch_l2(const void* ptr) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
-}
-
 struct GatherArgs {
   const void* k_pool;
   const void* v_pool;
@@ -223,18 +219,9 @@ gather_rope_kernel(const GatherArgs a) {
       else rope_sincos(delta, theta[e], &sn[e], &cs[e]);
     }
 
-    // the next token of the run, when it lies in the same shot, is the next pool row: its lines are
-    // asked for now (L2 prefetch), so that a warp has two tokens' worth of loads on their way
-    const bool next_in_shot = tt + 1 < kRun && p + 1 < o_next && p + 1 < a.ctx_cap;
     for (int l = 0; l < a.n_layers_call; ++l) {
       const long long src = (long long)(a.layer_begin + l) * layer_stride_pool + src_tok * row_vecs;
       const long long dst = ((long long)b * a.n_layers_call + l) * layer_stride_ctx + p * row_vecs;
-      if (next_in_shot) {
-        for (int i = lane * 8; i < row_vecs; i += 256) {          // one prefetch per 128-byte line of the row
-          prefetch_l2(kp + src + row_vecs + i);
-          if (with_v) prefetch_l2(vp + src + row_vecs + i);
-        }
-      }
       // K: rotate pairs.  unit = head * HALF_V + column; lane stride 32 keeps the column.
       for (int unit = lane; unit < pair_units; unit += 64) {
         const int unit2 = unit + 32;

@@ -24,7 +24,7 @@ class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
                  overlap: bool = False, fused: bool = False, entropy_overlap: bool = False,
-                 vpool: bool = False, device="cuda"):
+                 vpool: Optional[bool] = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
@@ -40,7 +40,12 @@ class ReusePath:
         self.ctx_off = torch.empty((batch, k + 1), dtype=torch.int64, device=device)
         self.chunks = [(lb, min(self.nl, lb + self.lpc)) for lb in range(0, self.nl, self.lpc)]
         self.fused = bool(fused)
-        self.vpool = bool(vpool) and not self.fused
+        if vpool is None:
+            # measured choice: a cache that stays in L2 between the gather and the attention (a single
+            # layer of one query) is cheapest to read in full; anything larger is better off with the
+            # K-only cache, whose gather moves half the bytes
+            vpool = batch * self.lpc * self.ctx_cap * 2 * hkv * d * (4 if model.dtype == ab.F32 else 2) > (128 << 20)
+        self.vpool = bool(vpool) and not self.fused and model.dtype != ab.F32
         self.overlap = bool(overlap) and len(self.chunks) > 1 and not self.fused
         n_ctx = batch * self.lpc * self.ctx_cap * hkv * d
         n_buf = 0 if self.fused else (2 if self.overlap else 1)     # the fused variant has no assembled cache
@@ -86,15 +91,17 @@ class ReusePath:
         ab.adapshot_assemble_kv(self.model, self.pool, self.sel_idx, layer_begin, layer_end,
                                 k_ctx, v_ctx, self.ctx_cap, self.ctx_off, self.status, flags=flags)
 
-    def attend(self, q, kq, vq, out, layer_begin: int, layer_end: int, buf: int = 0):
+    def attend(self, q, kq, vq, out, layer_begin: int, layer_end: int, buf: int = 0, probes=None):
+        """Attention of the probes (default: all of them; a sub-list must be ascending) over the cache."""
         k_ctx, v_ctx = self.ctx_views(layer_end - layer_begin, buf)
+        probes = self.probes if probes is None else list(probes)
         if self.vpool:
             ab.adapshot_query_attn_vpool(self.model, self.pool, self.sel_idx, k_ctx, self.ctx_cap, self.ctx_off,
-                                         self.probes, q, kq, vq, layer_begin, layer_end, out, None,
+                                         probes, q, kq, vq, layer_begin, layer_end, out, None,
                                          self.ws_attn, self.status)
             return
         ab.adapshot_query_attn(self.model, k_ctx, v_ctx, self.ctx_cap, self.ctx_off,
-                               self.k, self.probes, q, kq, vq, layer_begin, layer_end, out, None,
+                               self.k, probes, q, kq, vq, layer_begin, layer_end, out, None,
                                self.ws_attn, self.status)
 
     def attend_fused(self, q, kq, vq, out, layer_begin: int, layer_end: int):
