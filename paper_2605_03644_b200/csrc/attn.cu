@@ -863,12 +863,11 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // ----------------------------------------------- V tiles straight from the pool, stitched by TMA
     // Eq. 7 corrects K only, so V needs no assembled copy.  The 128 context positions of a tile map
     // to a few runs of consecutive pool rows (one per selected shot the tile touches): the lanes look
-    // the positions up and mark where a run ends; every run is brought as power-of-two boxes (maps with
-    // 128, 64, ..., 1-row boxes over the pool; a box may start at any row, its shared-memory address only
-    // has to be 128-byte aligned), one box per lane, all found before the stage is waited for.
-    // Positions beyond the context continue the last run (their P is exactly zero; rows outside the
-    // pool arrive as zeros), so every tile delivers the same number of bytes to its barrier.  The
-    // probe's own tokens are one run of the own-token tensor.
+    // the positions up and mark where a run ends; every run is brought as one or two power-of-two boxes
+    // (maps with 128, 64, ..., 1-row boxes over the pool; a box may start at any row, its shared-memory
+    // address only has to be 128-byte aligned), one box per lane, all found before the stage is waited
+    // for.  Positions beyond the context continue the last run (their P is exactly zero; rows outside
+    // the pool arrive as zeros).  The probe's own tokens are one run of the own-token tensor.
     int* rows_s = reinterpret_cast<int*>(base_ptr + SM::kOffRows);
     uint32_t tv = 0;
     bool ok = true;
@@ -940,10 +939,14 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const bool last = lane == 31 && q4 == 3;
             brk[q4] = __ballot_sync(0xffffffffu, last || nxt != r[q4] + 1);
           }
-          // the run ends as one 128-bit mask in every lane; lane j then finds the j-th box on its own:
-          // boxes are numbered run by run, a run of n rows gives popcount(n) boxes, largest first
+          // the run ends as one 128-bit mask in every lane; lane j then finds the j-th box on its own.
+          // A run of n rows takes the largest power-of-two box that fits, once from its first row and,
+          // unless n is that power of two, once more ending at its last row: the two overlap, both write
+          // the same values there, and no run needs more than two copy instructions (the copy engine's
+          // time goes with the number of instructions, not with the bytes)
           __syncwarp();
           int my_pidx = -1, my_row = 0, my_lg = 0, n_boxes = 0;
+          uint32_t tile_bytes = 0;                 // what the boxes deliver in all (overlaps are copied twice)
           {
             int pidx = 0;
             while (pidx < kTileN) {
@@ -953,15 +956,15 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (word != 0) { e += __ffs(word) - 1; break; }
                 e = (e | 31) + 1;
               }
-              int n = e - pidx + 1;
-              int off = 0;
-              while (n > 0) {
-                const int lg = 31 - __clz(n);      // the largest power-of-two box that fits
-                if (n_boxes == lane) { my_pidx = pidx + off; my_lg = lg; }
+              const int n = e - pidx + 1;
+              const int lg = 31 - __clz(n);        // the largest power-of-two box that fits
+              if (n_boxes == lane) { my_pidx = pidx; my_lg = lg; }
+              ++n_boxes;
+              if (n > (1 << lg)) {                 // the rest of the run: the same box once more, ending at the run's end
+                if (n_boxes == lane) { my_pidx = e + 1 - (1 << lg); my_lg = lg; }
                 ++n_boxes;
-                off += 1 << lg;
-                n -= 1 << lg;
               }
+              tile_bytes += (n > (1 << lg) ? 2u : 1u) * ((uint32_t)SUB << (lg + 7));
               pidx = e + 1;
             }
           }
@@ -969,7 +972,7 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           // (tiles of more than 32 boxes - many one-token shots - take further rounds of the same walk)
           if (lane == 0) {
             ok = mbar_wait(bar(kBarVEmpty + sv), ((tv / VS) & 1) ^ 1, abort_flag);
-            if (ok) mbar_arrive_expect_tx(bar(kBarVFull + sv), kTileBytes);
+            if (ok) mbar_arrive_expect_tx(bar(kBarVFull + sv), tile_bytes);
           }
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) break;
@@ -989,13 +992,13 @@ attn_main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (word != 0) { e += __ffs(word) - 1; break; }
                 e = (e | 31) + 1;
               }
-              int n = e - pidx + 1, off = 0;
-              while (n > 0) {
-                const int lg = 31 - __clz(n);
-                if (idx == round * 32 + lane) { bp = pidx + off; bl = lg; }
+              const int n = e - pidx + 1;
+              const int lg = 31 - __clz(n);
+              if (idx == round * 32 + lane) { bp = pidx; bl = lg; }
+              ++idx;
+              if (n > (1 << lg)) {
+                if (idx == round * 32 + lane) { bp = e + 1 - (1 << lg); bl = lg; }
                 ++idx;
-                off += 1 << lg;
-                n -= 1 << lg;
               }
               pidx = e + 1;
             }

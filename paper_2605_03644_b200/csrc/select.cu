@@ -20,6 +20,10 @@ __device__ __forceinline__ double key_score(unsigned long long k) { return ads_k
 // keys_out set (pools that the rank kernel handles) the warp also forms |q_b| from the values
 // it loads anyway and writes the sort key of cos(q_b, e_i) in place of the dot product, so
 // that the ranking kernel's CTAs do not each redo N fp64 divisions.
+// NV > 0: E = 128 NV, the row is widened to fp64 once and kept in registers for all B queries
+// (the fp32 -> fp64 conversions, not the fp64 FMAs, are what a row-times-many-queries pass pays for);
+// NV = 0: any E.
+template <int NV>
 __global__ void __launch_bounds__(256)
 cosine_dots_kernel(const float* __restrict__ emb, const float* __restrict__ q_emb, int N, int E,
                    int B, double* __restrict__ dots, double* __restrict__ enorm, int keys_out) {
@@ -27,8 +31,42 @@ cosine_dots_kernel(const float* __restrict__ emb, const float* __restrict__ q_em
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= N) return;
   const float* e = emb + (long long)row * E;
-  const bool vec_ok = (E & 3) == 0;
   double nn = 0.0;
+  if constexpr (NV > 0) {
+    double ev[4 * NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const float4 v = *reinterpret_cast<const float4*>(e + lane * 4 + 128 * i);
+      ev[4 * i] = v.x; ev[4 * i + 1] = v.y; ev[4 * i + 2] = v.z; ev[4 * i + 3] = v.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 4 * NV; ++j) nn += ev[j] * ev[j];
+    nn = warp_sum(nn);
+    if (lane == 0) enorm[row] = sqrt(nn);
+    for (int b = 0; b < B; ++b) {
+      const float* q = q_emb + (long long)b * E;
+      double acc = 0.0, qq = 0.0;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const float4 w = __ldg(reinterpret_cast<const float4*>(q + lane * 4 + 128 * i));
+        const double w0 = w.x, w1 = w.y, w2 = w.z, w3 = w.w;
+        acc += ev[4 * i] * w0 + ev[4 * i + 1] * w1 + ev[4 * i + 2] * w2 + ev[4 * i + 3] * w3;
+        if (keys_out) qq += w0 * w0 + w1 * w1 + w2 * w2 + w3 * w3;
+      }
+      acc = warp_sum(acc);
+      if (keys_out) {
+        qq = warp_sum(qq);
+        if (lane == 0) {
+          const double den = sqrt(qq) * sqrt(nn);
+          reinterpret_cast<unsigned long long*>(dots)[(long long)b * N + row] = desc_key(den > 0.0 ? acc / den : 0.0);
+        }
+      } else if (lane == 0) {
+        dots[(long long)b * N + row] = acc;
+      }
+    }
+    return;
+  }
+  const bool vec_ok = (E & 3) == 0;
   if (vec_ok) {
     for (int i = lane * 4; i < E; i += 128) {
       float4 v = *reinterpret_cast<const float4*>(e + i);
@@ -308,8 +346,14 @@ extern "C" int adapshot_select(const adapshot_pool_t* pool, const float* q_emb, 
   }
 
   const int warps_per_block = 8;
-  cosine_dots_kernel<<<(N + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
-      pool->emb, q_emb, N, E, B, dots, enorm, N <= kRankMaxN ? 1 : 0);
+  const unsigned cgrid = (unsigned)((N + warps_per_block - 1) / warps_per_block);
+  const int keys_out = N <= kRankMaxN ? 1 : 0;
+  if (E == 1024)
+    cosine_dots_kernel<8><<<cgrid, warps_per_block * 32, 0, st>>>(pool->emb, q_emb, N, E, B, dots, enorm, keys_out);
+  else if (E == 128)
+    cosine_dots_kernel<1><<<cgrid, warps_per_block * 32, 0, st>>>(pool->emb, q_emb, N, E, B, dots, enorm, keys_out);
+  else
+    cosine_dots_kernel<0><<<cgrid, warps_per_block * 32, 0, st>>>(pool->emb, q_emb, N, E, B, dots, enorm, keys_out);
   if (ads_launch_status() != ADAPSHOT_OK) return ADAPSHOT_ECUDA;
 
   if (N <= kRankMaxN) {
