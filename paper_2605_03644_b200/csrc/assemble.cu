@@ -117,8 +117,10 @@ struct GatherArgs {
 // 128-thread CTAs of at most 88 registers: small enough to be co-resident with a persistent
 // attention CTA (which leaves about 11.7 K registers and 1.5 KB of shared memory per SM), so
 // that the gather of the next layer chunk can run under the attention of the current one.
-template <typename T, int D>
-__global__ void __launch_bounds__(128, 6)
+// WITH_V = false: the K-only form (V is taken from the pool by its consumer); it keeps two layers'
+// loads in flight and takes the registers for that (five CTAs per SM instead of six).
+template <typename T, int D, bool WITH_V>
+__global__ void __launch_bounds__(128, WITH_V ? 6 : 5)
 gather_rope_kernel(const GatherArgs a) {
   constexpr int EPV = Vec16<T>::N;                 // elements per 16-byte vector
   constexpr int VPH = D / EPV;                     // vectors per head row
@@ -142,7 +144,7 @@ gather_rope_kernel(const GatherArgs a) {
   const uint4* vp = static_cast<const uint4*>(a.v_pool);
   uint4* kc = static_cast<uint4*>(a.k_ctx);
   uint4* vc = static_cast<uint4*>(a.v_ctx);
-  const bool with_v = vc != nullptr;               // a K-only cache: V is read from the pool by its consumer
+  constexpr bool with_v = WITH_V;
 
   // A warp takes a run of kRun consecutive destination tokens of one query.  The plan lookup
   // (which selected shot covers the position) is a dependent chain of global loads, so it is
@@ -219,39 +221,58 @@ gather_rope_kernel(const GatherArgs a) {
       else rope_sincos(delta, theta[e], &sn[e], &cs[e]);
     }
 
-    for (int l = 0; l < a.n_layers_call; ++l) {
+    // rotates one pair unit (vector j of the low half of a head with vector j of the high half) and stores it
+    auto rot_store = [&](const uint4& lo_v, const uint4& hi_v, long long d0) {
+      float x[EPV], y[EPV], xr[EPV], yr[EPV];
+      Vec16<T>::unpack(lo_v, x); Vec16<T>::unpack(hi_v, y);
+#pragma unroll
+      for (int e = 0; e < EPV; ++e) {
+        xr[e] = x[e] * cs[e] - y[e] * sn[e];
+        yr[e] = y[e] * cs[e] + x[e] * sn[e];
+      }
+      kc[d0] = Vec16<T>::pack(xr);
+      kc[d0 + HALF_V] = Vec16<T>::pack(yr);
+    };
+    int l_first = 0;
+    if (!with_v) {
+      // K alone: the loads of two layers are issued before either is rotated, so that a warp keeps as
+      // many bytes on their way as it does when it also copies V
+      for (; l_first + 1 < a.n_layers_call; l_first += 2) {
+        const long long srcA = (long long)(a.layer_begin + l_first) * layer_stride_pool + src_tok * row_vecs;
+        const long long srcB = srcA + layer_stride_pool;
+        const long long dstA = ((long long)b * a.n_layers_call + l_first) * layer_stride_ctx + p * row_vecs;
+        const long long dstB = dstA + layer_stride_ctx;
+        for (int unit = lane; unit < pair_units; unit += 64) {
+          const int unit2 = unit + 32;
+          const bool two = unit2 < pair_units;
+          const int o0 = (unit / HALF_V) * VPH + jcol, o1 = (unit2 / HALF_V) * VPH + jcol;
+          const uint4 z = make_uint4(0, 0, 0, 0);
+          const uint4 aLo0 = kp[srcA + o0], aHi0 = kp[srcA + o0 + HALF_V];
+          const uint4 bLo0 = kp[srcB + o0], bHi0 = kp[srcB + o0 + HALF_V];
+          const uint4 aLo1 = two ? kp[srcA + o1] : z, aHi1 = two ? kp[srcA + o1 + HALF_V] : z;
+          const uint4 bLo1 = two ? kp[srcB + o1] : z, bHi1 = two ? kp[srcB + o1 + HALF_V] : z;
+          rot_store(aLo0, aHi0, dstA + o0);
+          rot_store(bLo0, bHi0, dstB + o0);
+          if (two) {
+            rot_store(aLo1, aHi1, dstA + o1);
+            rot_store(bLo1, bHi1, dstB + o1);
+          }
+        }
+      }
+    }
+    for (int l = l_first; l < a.n_layers_call; ++l) {
       const long long src = (long long)(a.layer_begin + l) * layer_stride_pool + src_tok * row_vecs;
       const long long dst = ((long long)b * a.n_layers_call + l) * layer_stride_ctx + p * row_vecs;
       // K: rotate pairs.  unit = head * HALF_V + column; lane stride 32 keeps the column.
       for (int unit = lane; unit < pair_units; unit += 64) {
         const int unit2 = unit + 32;
         const bool two = unit2 < pair_units;
-        const int h0 = unit / HALF_V, h1 = unit2 / HALF_V;
-        const long long a0 = src + h0 * VPH + jcol, a1 = src + h1 * VPH + jcol;
-        uint4 lo0 = kp[a0], hi0 = kp[a0 + HALF_V];
+        const int o0 = (unit / HALF_V) * VPH + jcol, o1 = (unit2 / HALF_V) * VPH + jcol;
+        const uint4 lo0 = kp[src + o0], hi0 = kp[src + o0 + HALF_V];
         uint4 lo1 = make_uint4(0, 0, 0, 0), hi1 = lo1;
-        if (two) { lo1 = kp[a1]; hi1 = kp[a1 + HALF_V]; }
-        float x[EPV], y[EPV], xr[EPV], yr[EPV];
-        Vec16<T>::unpack(lo0, x); Vec16<T>::unpack(hi0, y);
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) {
-          xr[e] = x[e] * cs[e] - y[e] * sn[e];
-          yr[e] = y[e] * cs[e] + x[e] * sn[e];
-        }
-        const long long d0 = dst + h0 * VPH + jcol;
-        kc[d0] = Vec16<T>::pack(xr);
-        kc[d0 + HALF_V] = Vec16<T>::pack(yr);
-        if (two) {
-          Vec16<T>::unpack(lo1, x); Vec16<T>::unpack(hi1, y);
-#pragma unroll
-          for (int e = 0; e < EPV; ++e) {
-            xr[e] = x[e] * cs[e] - y[e] * sn[e];
-            yr[e] = y[e] * cs[e] + x[e] * sn[e];
-          }
-          const long long d1 = dst + h1 * VPH + jcol;
-          kc[d1] = Vec16<T>::pack(xr);
-          kc[d1 + HALF_V] = Vec16<T>::pack(yr);
-        }
+        if (two) { lo1 = kp[src + o1]; hi1 = kp[src + o1 + HALF_V]; }
+        rot_store(lo0, hi0, dst + o0);
+        if (two) rot_store(lo1, hi1, dst + o1);
       }
       // V: plain copy, four vectors in flight per lane
       for (int i = lane; with_v && i < row_vecs; i += 128) {
@@ -287,7 +308,8 @@ int launch_gather(GatherArgs a, cudaStream_t st) {
   // layer per call), several waves when every run walks several layers
   const long long max_blocks = a.n_layers_call == 1 ? n_sm * 6 : n_sm * 16 * 4;
   if (blocks > max_blocks) blocks = max_blocks;
-  gather_rope_kernel<T, D><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
+  if (a.v_ctx != nullptr) gather_rope_kernel<T, D, true><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
+  else gather_rope_kernel<T, D, false><<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(a);
   return ads_launch_status();
 }
 

@@ -29,12 +29,12 @@ __device__ __forceinline__ EntState ent_merge(EntState a, EntState b) {
   return r;
 }
 
-// Adds N logits to a state.  The exponentials run in the log2 domain: y = (x - m) log2(e) is one
-// FMA, e = 2^y one MUFU operation, and t accumulates e * y (converted to natural units once, when the
-// group of N is done).  y is clamped at -2^20 so that a logit of -inf gives e = 0 and e * y = -0, not NaN.
+// Adds N logits to a state.  d = x - m is formed exactly (the row maximum itself gives d = 0 and
+// e = 1), e = 2^(d log2 e) is one multiply and one MUFU operation, t accumulates e * d.  d is clamped
+// at -1e30 so that a logit of -inf gives e = 0 and e * d = -0, not NaN.
 template <int N>
 __device__ __forceinline__ void ent_accumulate(EntState& st, const float (&x)[N]) {
-  constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+  constexpr float kLog2e = 1.4426950408889634f;
   float vm = x[0];
 #pragma unroll
   for (int i = 1; i < N; ++i) vm = fmaxf(vm, x[i]);
@@ -44,18 +44,17 @@ __device__ __forceinline__ void ent_accumulate(EntState& st, const float (&x)[N]
     st.s *= e;
     st.m = vm;
   }
-  const float neg_m2 = -st.m * kLog2e;
-  float s_add = 0.f, t2_add = 0.f;
+  float s_add = 0.f, t_add = 0.f;
 #pragma unroll
   for (int i = 0; i < N; ++i) {
-    const float y = fmaxf(fmaf(x[i], kLog2e, neg_m2), -1048576.f);
+    const float d = fmaxf(x[i] - st.m, -1.0e30f);
     float e;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(y));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(d * kLog2e));
     s_add += e;
-    t2_add = fmaf(e, y, t2_add);
+    t_add = fmaf(e, d, t_add);
   }
   st.s += s_add;
-  st.t = fmaf(t2_add, kLn2, st.t);
+  st.t += t_add;
 }
 
 __device__ __forceinline__ EntState ent_warp_reduce(EntState st) {
