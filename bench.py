@@ -111,7 +111,11 @@ SUB_WORKLOADS = ("cfg2", "cfg3")   # reported beside it in the default run, each
 # average, so the traffic grows in proportion.  None = no capture of the kernel as it stands.
 NCU_TRAFFIC = {
     # workload: (attn_main bytes per captured launch, layers x queries in that capture,
-    #            gather bytes per captured launch, layers x queries in that capture)
+    #            gather bytes per captured launch, layers x queries in that capture), for the variant
+    #            that `--variant auto` picks for the workload
+    "cfg2": (102.0e6, 1, 119.7e6, 1),             # profiles/attn_main_kernel_cfg2.md, profiles/gather_rope_kernel.md
+    "cfg3": (2.2323e9, 16, 2.110e9, 16),          # profiles/attn_main_kernel_cfg3_2layers.md (2 layers x 8 queries, K-only cache)
+    "cfg5": (2.050e9, 4, 1.0684e9, 4),            # profiles/attn_main_and_gather_cfg5_1layer_4queries.md (K-only cache)
 }
 
 
@@ -152,12 +156,15 @@ def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e
 
 
 def choose_variant(w: wl.Workload, ctx_cap: int, variant: str = "auto", layers_per_call: int = 0):
-    """(vpool, layers per call) of a run.  auto: the K-only cache (V taken from the pool) when the full cache of
-    one call would be larger than L2, the full cache otherwise (the rule of ReusePath(vpool=None))."""
+    """(vpool, layers per call) of a run.  auto (the rule of ReusePath(vpool=None)): the K-only cache, V taken
+    from the pool, when the full cache of one call would be larger than L2 and a KV head has at most 1024 query
+    rows (with more rows the gather is a small share of the call and the dearer V tiles cost more than half a
+    gather saves); the full cache otherwise."""
     vpool = variant == "vpool"
     if variant == "auto":
         lpc_full = layers_per_call or layers_per_call_for(w, ctx_cap)
-        vpool = w.batch * lpc_full * ctx_cap * w.bytes_per_token_layer > (128 << 20)
+        vpool = (w.batch * lpc_full * ctx_cap * w.bytes_per_token_layer > (128 << 20)
+                 and w.t_q * w.group <= 1024)
     return vpool, (layers_per_call or layers_per_call_for(w, ctx_cap, k_only=vpool))
 
 
@@ -519,7 +526,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
         counts["attn_kv_bytes"] / (peaks["hbm_gbs"] * 1e9)
     traffic_attn = traffic_gather = None
     cap = NCU_TRAFFIC.get(w.name)
-    if cap is not None and not fused and not vpool and not args.layers and not args.queries and args.k_pos_mode == 0:
+    if cap is not None and args.variant == "auto" and not args.layers and not args.queries and args.k_pos_mode == 0:
         units_per_launch = path.lpc * w.batch
         if cap[0] is not None:
             traffic_attn = cap[0] / cap[1] * units_per_launch
@@ -669,6 +676,24 @@ def run_micro(args):
         fn = lambda: ab.adapshot_entropy(logits, H, args.tau, 1, fo, ws, st)
         nbytes = float(R) * V * logits.element_size()
         what = {"rows": R, "vocab": V, "logits_dtype": args.logits_dtype}
+    elif args.micro == "relevance":
+        # the attention-based selector (Sec. 4.2) over one layer of a workload's pool: tensor-core passes, bound
+        # by the exponentials (one per query row and pool key, twice)
+        w = wl.CONFIGS["cfg3" if args.workload == "default" else args.workload]
+        pool = wl.make_pool(w, dev, n_layers=1)
+        so = torch.from_numpy(pool["shot_off"]).to(dev)
+        dpool = ab.Pool(so, pool["k"], pool["v"], pool["emb"])
+        model = ab.make_model(1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.rope_base)
+        q = torch.randn(w.batch, w.t_q, w.n_q_heads, w.head_dim, generator=g, device=dev).to(torch.bfloat16)
+        sel = torch.empty((w.batch, w.k), dtype=torch.int32, device=dev)
+        ws = torch.empty(max(256, ab.adapshot_select_attn_workspace_bytes(model, dpool, w.batch, w.t_q, w.k)),
+                         dtype=torch.uint8, device=dev)
+        fn = lambda: ab.adapshot_select_attn(model, dpool, 0, q, w.k, sel, None, ws, st)
+        rows = float(w.batch) * w.t_q * w.n_q_heads
+        flops = 2.0 * 2.0 * rows * pool["pool_tokens"] * w.head_dim            # two passes of Q K^T
+        nbytes = 2.0 * pool["pool_tokens"] * w.n_kv_heads * w.head_dim * 2     # the layer's K, twice
+        what = {"workload": w.name, "pool_tokens": int(pool["pool_tokens"]), "query_rows": rows,
+                "algorithmic_flops": flops, "exponentials": 2.0 * rows * pool["pool_tokens"]}
     else:
         w = wl.CONFIGS[HEADLINE if args.workload == "default" else args.workload]
         n_shots = int(wl.shot_lengths(w).size)
@@ -690,6 +715,11 @@ def run_micro(args):
     if st.item() != 0:
         raise SystemExit(f"device status {st.item()}")
     gbs = nbytes / (ms * 1e-3) / 1e9
+    if args.micro == "relevance":
+        what["achieved_tflops"] = what["algorithmic_flops"] / (ms * 1e-3) / 1e12
+        what["frac_of_bf16_peak"] = what["achieved_tflops"] / peaks["bf16_tflops"]
+        # 16 exponentials per clock and SM at the clock the sampler saw
+        what["exp_per_s"] = what["exponentials"] / (ms * 1e-3)
     print(json.dumps({"micro": args.micro, **what, "algorithmic_bytes": nbytes, "ms_per_call": ms, "steps": steps,
                       "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
                       "peak_source": f"of {peaks['source']}", "clocks": clocks.summary(),
@@ -768,7 +798,7 @@ def main():
                     help="replay the pass as one CUDA graph (auto: single-layer workloads)")
     ap.add_argument("--entropy-overlap", action="store_true",
                     help="run the entropy probe on a side stream beside the pass instead of after the attention")
-    ap.add_argument("--micro", default=None, choices=["entropy", "select"],
+    ap.add_argument("--micro", default=None, choices=["entropy", "select", "relevance"],
                     help="time one HBM-bound step alone on a bandwidth-bound input and print its own JSON line")
     ap.add_argument("--rows", type=int, default=2048, help="--micro entropy: logit rows")
     ap.add_argument("--vocab", type=int, default=128256, help="--micro entropy: vocabulary size")

@@ -28,6 +28,13 @@ constexpr int kTile = 128;            // query rows per M tile, keys per tile
 constexpr int kRelThreads = 192;      // warp 0 TMA, warp 1 MMA, warps 2-5 consumers (one thread per TMEM lane)
 constexpr int kKStages = 3;
 
+// 2^x by the hardware approximation (one MUFU operation, relative error about 2^-22; 2^-inf = 0)
+__device__ __forceinline__ float rel_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 struct RelParams {
   float* ml_part;               // pass 1 out: [unit][split][128][2] (max in log2 units, sum)
   const float* lse2;            // pass 2 in:  [unit][128] log2-sum-exp of every query row
@@ -136,7 +143,11 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256);
     tmem_relinquish();
   }
-  if (PASS == 2 && threadIdx.x >= 64) lse_s[threadIdx.x - 64] = p.lse2[(long long)unit * kTile + threadIdx.x - 64];
+  if (PASS == 2 && threadIdx.x >= 64) {
+    // rows of the M tile that do not exist get lse = +inf: their 2^(s c - lse) is exactly zero
+    const int c = threadIdx.x - 64;
+    lse_s[c] = c < min(kTile, p.rows - mt * kTile) ? p.lse2[(long long)unit * kTile + c] : INFINITY;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -203,7 +214,6 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;                      // TMEM lane: query row (pass 1) or key of the tile (pass 2)
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    const int rows_valid = min(kTile, p.rows - mt * kTile); // query rows of this M tile that exist
     float m_run = -1.0e30f, l_run = 0.f;
     bool ok = true;
     for (int i = 0; i < n_it; ++i) {
@@ -218,18 +228,24 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const long long key0 = (long long)(t0 + i) * kTile;
       if (PASS == 1) {
         const int limit = (int)min((long long)kTile, p.pool_tokens - key0);   // keys of this tile that exist
-        float mx = -INFINITY;
+        if (limit < kTile) {                       // only the pool's last tile: keys beyond it count as -inf
 #pragma unroll
-        for (int c = 0; c < kTile; ++c) mx = fmaxf(mx, c < limit ? s[c] : -INFINITY);
-        mx *= p.scale_log2;
+          for (int c = 0; c < kTile; ++c) s[c] = c < limit ? s[c] : -INFINITY;
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int c = 0; c < kTile; c += 8) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mx4[u] = fmax3(mx4[u], s[c + 2 * u], s[c + 2 * u + 1]);
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
         if (mx > m_run) {
-          l_run *= exp2f(m_run - mx);
+          l_run *= rel_ex2(m_run - mx);
           m_run = mx;
         }
         float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < kTile; ++c)
-          part[c & 3] += c < limit ? exp2f(fmaf(s[c], p.scale_log2, -m_run)) : 0.f;
+        for (int c = 0; c < kTile; ++c) part[c & 3] += rel_ex2(fmaf(s[c], p.scale_log2, -m_run));
         l_run += (part[0] + part[1]) + (part[2] + part[3]);
       } else {
         const long long key = key0 + r;
@@ -240,8 +256,7 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const float4 l4 = lse4[c4];                     // the same address for every lane: a broadcast
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            part[e] += 4 * c4 + e < rows_valid ? exp2f(fmaf(s[4 * c4 + e], p.scale_log2, -lv[e])) : 0.f;
+          for (int e = 0; e < 4; ++e) part[e] += rel_ex2(fmaf(s[4 * c4 + e], p.scale_log2, -lv[e]));
         }
         float v = (part[0] + part[1]) + (part[2] + part[3]);
         int id = -1;

@@ -43,8 +43,10 @@ class ReusePath:
         if vpool is None:
             # measured choice: a cache that stays in L2 between the gather and the attention (a single
             # layer of one query) is cheapest to read in full; anything larger is better off with the
-            # K-only cache, whose gather moves half the bytes
-            vpool = batch * self.lpc * self.ctx_cap * 2 * hkv * d * (4 if model.dtype == ab.F32 else 2) > (128 << 20)
+            # K-only cache, whose gather moves half the bytes - unless a KV head has so many query rows
+            # (more than 1024) that the gather is a small share of the call anyway
+            vpool = (batch * self.lpc * self.ctx_cap * 2 * hkv * d * (4 if model.dtype == ab.F32 else 2) > (128 << 20)
+                     and t_q * (hq // hkv) <= 1024)
         self.vpool = bool(vpool) and not self.fused and model.dtype != ab.F32
         self.overlap = bool(overlap) and len(self.chunks) > 1 and not self.fused
         n_ctx = batch * self.lpc * self.ctx_cap * hkv * d
