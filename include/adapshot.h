@@ -297,9 +297,14 @@ ADAPSHOT_API int adapshot_decode_attn(const adapshot_model_t* model, const void*
  *                 H[g*rows_per_group + j] <= tau, else -1   (int32 out, or NULL)
  *   logits [R][row_stride] fp32 or bf16 (dtype), row_stride in elements, rows
  *   16-byte aligned; one pass with a running maximum, fp32 accumulation.
+ *   A logit at or below -2^97 (about -1.6e29) counts as -inf: it adds nothing; a row
+ *   that holds nothing above it, and an all-NaN row, give H = 0.
  *   Limits: R a multiple of rows_per_group, rows_per_group <= 8192, and
- *   R * splits < 2^31 with splits = min(ceil(1184 / R), ceil(V / 4096)) (one CTA
- *   per row and split); ADAPSHOT_ESHAPE otherwise.                              */
+ *   R * splits < 2^31, where splits (one CTA per row and split) is the n in
+ *   1..min(64, ceil(V / 4096)) that minimises
+ *   ceil(R * n / 1184) * (ceil(V / n) + 1024); ADAPSHOT_ESHAPE otherwise.
+ *   Ask adapshot_entropy_workspace_bytes for the scratch size (12 bytes per row and
+ *   split, rounded up to 256).                                                   */
 ADAPSHOT_API size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V);
 ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V, int64_t row_stride,
                      float* H, float tau, int32_t rows_per_group, int32_t* first_ok,
@@ -329,9 +334,9 @@ ADAPSHOT_API int adapshot_entropy_subset(const void* logits, int32_t dtype, int3
  * and error codes as adapshot_entropy, minus `ws`: the per-split states live in
  * a fixed 192 KiB device array inside the library (one per GPU that loads it,
  * held until the process exits).
- *  - Limit: R * splits <= 16384 states, where splits = min(ceil(1184 / R),
- *    ceil(V / 4096)); larger requests return ADAPSHOT_ECAPACITY and launch
- *    nothing.  (Examples within the limit: 8 rows x 128256; 224 rows x 128256.)
+ *  - Limit: R <= 16384 rows; more return ADAPSHOT_ECAPACITY and launch nothing.
+ *    The rows are split as in adapshot_entropy, but never into more than
+ *    floor(16384 / R) slices each (the array holds 16384 states).
  *  - The first call on each device looks up the array's device address (with
  *    that device current); make that first call outside any stream capture.
  *  - The call allocates and frees nothing, on the host or the device.

@@ -29,32 +29,67 @@ __device__ __forceinline__ EntState ent_merge(EntState a, EntState b) {
   return r;
 }
 
-// Adds N logits to a state.  d = x - m is formed exactly (the row maximum itself gives d = 0 and
-// e = 1), e = 2^(d log2 e) is one multiply and one MUFU operation, t accumulates e * d.  d is clamped
-// at -1e30 so that a logit of -inf gives e = 0 and e * d = -0, not NaN.
+__device__ __forceinline__ float ent_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float ent_max3(float a, float b, float c) {   // one instruction on sm_100
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Logits at or below this value count as -inf: the loaders raise every logit to it (an exact
+// operation), so that x - m stays finite and e * (x - m) is -0, not NaN, where e underflows to 0.
+// -2^97 is exact in bf16 and in fp32.  A row that holds nothing above it has entropy 0 by
+// convention (entropy_finish_kernel).
+constexpr float kEntFloor = -1.5845632502852868e29f;
+constexpr uint32_t kEntFloorBf16x2 = 0xF000F000u;
+
+// Adds N logits (already raised to kEntFloor) to a state.  d = x - m is formed exactly (the row
+// maximum itself gives d = 0 and e = 1), e = 2^(d log2 e) is one multiply and one MUFU operation,
+// t accumulates e * d.  Pairs of logits go through the two-wide fp32 add / multiply / FMA forms,
+// which halves the instructions around the exponential.
 template <int N>
 __device__ __forceinline__ void ent_accumulate(EntState& st, const float (&x)[N]) {
   constexpr float kLog2e = 1.4426950408889634f;
   float vm = x[0];
+  {
+    int i = 1;
 #pragma unroll
-  for (int i = 1; i < N; ++i) vm = fmaxf(vm, x[i]);
+    for (; i + 1 < N; i += 2) vm = ent_max3(vm, x[i], x[i + 1]);
+    if (i < N) vm = fmaxf(vm, x[i]);
+  }
   if (vm > st.m) {
     float e = __expf(st.m - vm);
     st.t = st.s > 0.f ? (st.t + st.s * (st.m - vm)) * e : 0.f;
     st.s *= e;
     st.m = vm;
   }
-  float s_add = 0.f, t_add = 0.f;
+  if constexpr (N % 2 == 0) {
+    const float2 neg_m = make_float2(-st.m, -st.m);
+    const float2 l2e = make_float2(kLog2e, kLog2e);
+    float2 s2 = make_float2(0.f, 0.f), t2 = make_float2(0.f, 0.f);
 #pragma unroll
-  for (int i = 0; i < N; ++i) {
-    const float d = fmaxf(x[i] - st.m, -1.0e30f);
-    float e;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(d * kLog2e));
-    s_add += e;
-    t_add = fmaf(e, d, t_add);
+    for (int i = 0; i < N; i += 2) {
+      const float2 d = __fadd2_rn(make_float2(x[i], x[i + 1]), neg_m);
+      const float2 a = __fmul2_rn(d, l2e);
+      const float2 e = make_float2(ent_ex2(a.x), ent_ex2(a.y));
+      s2 = __fadd2_rn(s2, e);
+      t2 = __ffma2_rn(e, d, t2);
+    }
+    st.s += s2.x + s2.y;
+    st.t += t2.x + t2.y;
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const float d = x[i] - st.m;
+      const float e = ent_ex2(d * kLog2e);
+      st.s += e;
+      st.t = fmaf(e, d, st.t);
+    }
   }
-  st.s += s_add;
-  st.t += t_add;
 }
 
 __device__ __forceinline__ EntState ent_warp_reduce(EntState st) {
@@ -75,39 +110,57 @@ constexpr int kEntThreads = 256;
 // bound by the 65535 limit of the other grid dimensions).
 // partial[(r * n_split + s)] = state of slice s of row r.
 template <typename T>
-__global__ void __launch_bounds__(kEntThreads)
+__global__ void __launch_bounds__(kEntThreads, 6)
 entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride, int slice, int n_split,
                        float* __restrict__ partial) {
   constexpr int kVec = 16 / sizeof(T);
+  constexpr float kLog2e = 1.4426950408889634f;
   const int r = blockIdx.x / n_split, sp = blockIdx.x % n_split;
   const T* row = logits + (long long)r * row_stride;
   const int begin = sp * slice;
   const int end = min(V, begin + slice);
-  EntState st{-FLT_MAX, 0.f, 0.f};
+  EntState st{kEntFloor, 0.f, 0.f};    // every logit is at least the floor, so m starts there
 
-  const int vec_end = begin + ((end - begin) / kVec) * kVec;   // slice is a multiple of kVec
+  const int n_vec = (end - begin) / kVec;                        // slice is a multiple of kVec
   auto widen = [](const uint4& raw, float (&x)[kVec]) {
     if constexpr (sizeof(T) == 4) {
-      x[0] = __uint_as_float(raw.x); x[1] = __uint_as_float(raw.y);
-      x[2] = __uint_as_float(raw.z); x[3] = __uint_as_float(raw.w);
+      x[0] = fmaxf(__uint_as_float(raw.x), kEntFloor); x[1] = fmaxf(__uint_as_float(raw.y), kEntFloor);
+      x[2] = fmaxf(__uint_as_float(raw.z), kEntFloor); x[3] = fmaxf(__uint_as_float(raw.w), kEntFloor);
     } else {
       const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {   // bf16 -> fp32 is a 16-bit shift
-        x[2 * j] = __uint_as_float(w[j] << 16);
-        x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      for (int j = 0; j < 4; ++j) {   // the floor on both halves at once; bf16 -> fp32 is a 16-bit shift
+        uint32_t c;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(w[j]), "r"(kEntFloorBf16x2));
+        x[2 * j] = __uint_as_float(c << 16);
+        x[2 * j + 1] = __uint_as_float(c & 0xffff0000u);
       }
     }
   };
-  // four 16-byte loads in flight per thread: a CTA's 256 threads keep 16 KB on their way, which
-  // is what it takes to cover the DRAM latency at full bandwidth with a few CTAs per SM
+  // Four 16-byte loads per thread are kept in flight: a vector is copied out of its register,
+  // the load of the vector four steps ahead goes into that register at once, and only then is
+  // the copy worked on, so the memory system is never idle while a warp computes.  The host cuts
+  // rows into slices that are multiples of kEntSliceUnit, so that all but a row's last slice run
+  // in this loop alone.
   constexpr int kUnroll = 4;
-  constexpr int kStep = kEntThreads * kVec;
-  int i = begin + threadIdx.x * kVec;
-  for (; i + (kUnroll - 1) * kStep < vec_end; i += kUnroll * kStep) {
+  const uint4* vp = reinterpret_cast<const uint4*>(row + begin) + threadIdx.x;
+  const uint4* const vp_end = reinterpret_cast<const uint4*>(row + begin) + n_vec;
+  const int trips = n_vec / (kUnroll * kEntThreads);
+  if (trips > 0) {
     uint4 raw[kUnroll];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) raw[u] = __ldcs(reinterpret_cast<const uint4*>(row + i + u * kStep));
+    for (int u = 0; u < kUnroll; ++u) raw[u] = __ldcs(vp + u * kEntThreads);
+    for (int t = 1; t < trips; ++t) {
+      vp += kUnroll * kEntThreads;
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        float x[kVec];
+        widen(raw[u], x);
+        raw[u] = __ldcs(vp + u * kEntThreads);
+        ent_accumulate(st, x);
+      }
+    }
+    vp += kUnroll * kEntThreads;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       float x[kVec];
@@ -115,29 +168,46 @@ entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride
       ent_accumulate(st, x);
     }
   }
-  for (; i < vec_end; i += kStep) {
+  for (; vp < vp_end; vp += kEntThreads) {
     float x[kVec];
-    widen(__ldcs(reinterpret_cast<const uint4*>(row + i)), x);
+    widen(__ldcs(vp), x);
     ent_accumulate(st, x);
   }
-  for (int i = vec_end + threadIdx.x; i < end; i += kEntThreads) {   // ragged tail of the row
+  for (int i = begin + n_vec * kVec + threadIdx.x; i < end; i += kEntThreads) {   // ragged tail of the row
     float x[1];
-    if constexpr (sizeof(T) == 4) x[0] = row[i];
-    else x[0] = __bfloat162float(row[i]);
+    if constexpr (sizeof(T) == 4) x[0] = fmaxf(row[i], kEntFloor);
+    else x[0] = fmaxf(__bfloat162float(row[i]), kEntFloor);
     ent_accumulate(st, x);
   }
 
-  st = ent_warp_reduce(st);
-  __shared__ EntState sh[kEntThreads / 32];
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = st;
+  // CTA-wide merge: the maximum first; every thread then moves its (s, t) to it once, and what is
+  // left are plain sums (a butterfly of whole states would pay two exponentials per level)
+  __shared__ float sh_m[kEntThreads / 32], sh_s[kEntThreads / 32], sh_t[kEntThreads / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float M = st.m;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  if (lane == 0) sh_m[warp] = M;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    EntState v = threadIdx.x < kEntThreads / 32 ? sh[threadIdx.x] : EntState{-FLT_MAX, 0.f, 0.f};
-    v = ent_warp_reduce(v);
-    if (threadIdx.x == 0) {
-      float* o = partial + 3ll * ((long long)r * n_split + sp);
-      o[0] = v.m; o[1] = v.s; o[2] = v.t;
-    }
+  M = sh_m[0];
+#pragma unroll
+  for (int w = 1; w < kEntThreads / 32; ++w) M = fmaxf(M, sh_m[w]);
+  const float d = fmaxf(st.m - M, -1.0e30f);          // <= 0; the clamp keeps s * d finite
+  const float e = ent_ex2(d * kLog2e);
+  float ss = st.s * e, tt = fmaf(st.s, d, st.t) * e;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    tt += __shfl_xor_sync(0xffffffffu, tt, o);
+  }
+  if (lane == 0) { sh_s[warp] = ss; sh_t[warp] = tt; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ss = 0.f; tt = 0.f;
+#pragma unroll
+    for (int w = 0; w < kEntThreads / 32; ++w) { ss += sh_s[w]; tt += sh_t[w]; }
+    float* o = partial + 3ll * ((long long)r * n_split + sp);
+    o[0] = M; o[1] = ss; o[2] = tt;
   }
 }
 
@@ -159,7 +229,8 @@ entropy_finish_kernel(const float* __restrict__ partial, int n_split, int R, int
     }
     st = ent_warp_reduce(st);
     if (lane == 0) {
-      float h = st.s > 0.f ? logf(st.s) - st.t / st.s : 0.f;
+      // a maximum at the floor: the row holds nothing but -inf (or values that count as it)
+      float h = (st.s > 0.f && st.m > kEntFloor) ? logf(st.s) - st.t / st.s : 0.f;
       h = fmaxf(h, 0.f);
       H[r] = h;
       sh_h[j] = h;
@@ -237,17 +308,35 @@ entropy_subset_finish_kernel(const float* __restrict__ partial, int n_split, int
 }
 
 // A fixed figure rather than the SM count of the current device, so that the workspace size
-// can be asked for without a device and does not change from one GPU to another.
-constexpr int kEntTargetCtas = 1184;
+// can be asked for without a device and does not change from one GPU to another: one resident
+// wave of 256-thread CTAs at 40 registers (six per SM) on 148 SMs.
+constexpr int kEntTargetCtas = 888;
+constexpr int kEntSliceUnit = 8192;      // entries: what a CTA's unrolled loop takes per trip (bf16)
+constexpr int kEntCtaOverhead = 2048;    // fixed cost of a CTA (start, state merge, store) in entries
 
-int ent_splits(int R, int V) {
-  // about kEntTargetCtas CTAs in all (one resident wave of 256-thread CTAs on 148 SMs), each slice
-  // at least 4096 entries
-  int want = (kEntTargetCtas + R - 1) / R;
-  int max_by_len = (V + 4095) / 4096;
-  int s = want < max_by_len ? want : max_by_len;
-  return s < 1 ? 1 : s;
+// Rows are cut into slices of j * kEntSliceUnit entries (the last one shorter).  A call's CTAs run
+// in ceil(R * n / kEntTargetCtas) waves of about equal length (slice + overhead), so the j that
+// minimises waves * (slice + overhead) is taken: 2048 rows of 128 256 run as 2 slices each (4.6
+// waves) rather than whole (2.3 waves, the third one a third full), 224 rows as 3 slices (one wave).  `max_states` bounds R * n (the fixed scratch of the static entry point).
+struct EntSplit { int slice, n; };
+EntSplit ent_split(int R, int V, long long max_states = 0x7fffffffll) {
+  const int j_max = (V + kEntSliceUnit - 1) / kEntSliceUnit;     // j_max units: the row in one piece
+  EntSplit best{j_max * kEntSliceUnit, 1};
+  double best_cost = 0.0;
+  for (int j = j_max; j >= 1; --j) {
+    const int slice = j * kEntSliceUnit;
+    const int n = (V + slice - 1) / slice;
+    if (n > 64 || (long long)R * n > max_states) break;          // n only grows as j falls
+    const long long waves = ((long long)R * n + kEntTargetCtas - 1) / kEntTargetCtas;
+    const double cost = (double)waves * (slice + kEntCtaOverhead);
+    if (j == j_max || cost < best_cost) {
+      best = EntSplit{slice, n};
+      best_cost = cost;
+    }
+  }
+  return best;
 }
+int ent_splits(int R, int V) { return ent_split(R, V).n; }
 
 }  // namespace
 
@@ -272,10 +361,8 @@ extern "C" int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, in
   if (ws_bytes < adapshot_entropy_workspace_bytes(R, V)) return ADAPSHOT_ECAPACITY;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int n_split = ent_splits(R, V);
-  const int vec = 16 / (int)es;
-  int slice = (V + n_split - 1) / n_split;
-  slice = (slice + vec - 1) / vec * vec;
+  const EntSplit cut = ent_split(R, V);
+  const int n_split = cut.n, slice = cut.slice;
   const unsigned grid = (unsigned)((long long)R * n_split);
   float* partial = static_cast<float*>(ws);
   if (dtype == ADAPSHOT_F32)
@@ -310,10 +397,8 @@ extern "C" int adapshot_entropy_subset(const void* logits, int32_t dtype, int32_
   if (ws_bytes < adapshot_entropy_workspace_bytes(R, V)) return ADAPSHOT_ECAPACITY;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int n_split = ent_splits(R, V);
-  const int vec = 16 / (int)es;
-  int slice = (V + n_split - 1) / n_split;
-  slice = (slice + vec - 1) / vec * vec;
+  const EntSplit cut = ent_split(R, V);
+  const int n_split = cut.n, slice = cut.slice;
   const unsigned grid = (unsigned)((long long)R * n_split);
   float* partial = static_cast<float*>(ws);
   const int renorm = (int)(flags & 1u);
@@ -382,17 +467,15 @@ extern "C" int adapshot_entropy_static(const void* logits, int32_t dtype, int32_
   if ((long long)R * ent_splits(R, V) > 0x7fffffffll) return ADAPSHOT_ESHAPE;
   const size_t es = dtype == ADAPSHOT_F32 ? 4 : 2;
   if (!ads_aligned16(logits) || (row_stride * es) % 16 != 0) return ADAPSHOT_EALIGN;
-  const int n_split = ent_splits(R, V);
-  if ((long long)R * n_split > kStaticEntStates) return ADAPSHOT_ECAPACITY;   // beyond the fixed array
+  if (R > kStaticEntStates) return ADAPSHOT_ECAPACITY;   // beyond the fixed array
+  const EntSplit cut = ent_split(R, V, kStaticEntStates);
+  const int n_split = cut.n, slice = cut.slice;
 
   float* partial = nullptr;
   const int rc = static_scratch_for_current_device(&partial);
   if (rc != ADAPSHOT_OK) return rc;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int vec = 16 / (int)es;
-  int slice = (V + n_split - 1) / n_split;
-  slice = (slice + vec - 1) / vec * vec;
   const unsigned grid = (unsigned)((long long)R * n_split);
   // every (row, split) state this call reads is written by the first kernel, so
   // nothing in the shared array has to start at zero

@@ -26,7 +26,9 @@ using namespace sm100;
 
 constexpr int kTile = 128;            // query rows per M tile, keys per tile
 constexpr int kRelThreads = 192;      // warp 0 TMA, warp 1 MMA, warps 2-5 consumers (one thread per TMEM lane)
-constexpr int kKStages = 3;
+// K tiles in flight per CTA: two CTAs share an SM (96 KB each at d = 128), so that one's consumers
+// work while the other's wait for a score tile
+template <int D> constexpr int kKStages = D == 128 ? 2 : 4;
 
 // 2^x by the hardware approximation (one MUFU operation, relative error about 2^-22; 2^-inf = 0)
 __device__ __forceinline__ float rel_ex2(float x) {
@@ -84,14 +86,14 @@ __global__ void __launch_bounds__(256) rel_token_shot_kernel(const long long* __
   tok_shot[t] = lo;
 }
 
-enum RelBar { kRQFull = 0, kRKFull = 1, kRKEmpty = 4, kRSFull = 7, kRSEmpty = 9, kRDrain = 11, kRNumBars = 12 };
+enum RelBar { kRQFull = 0, kRKFull = 1, kRKEmpty = 5, kRSFull = 9, kRSEmpty = 11, kRDrain = 13, kRNumBars = 14 };
 
 template <int D>
 struct RelSmem {
   static constexpr uint32_t kTileBytes = (D / 64) * 16384u;
   static constexpr uint32_t kOffQ = 0;
   static constexpr uint32_t kOffK = kTileBytes;
-  static constexpr uint32_t kOffBar = kOffK + kKStages * kTileBytes;
+  static constexpr uint32_t kOffBar = kOffK + kKStages<D> * kTileBytes;
   static constexpr uint32_t kOffLse = kOffBar + 128;
   static constexpr uint32_t kTotal = kOffLse + 512 + 1024;      // + alignment slack
 };
@@ -99,11 +101,12 @@ struct RelSmem {
 // grid (B * n_mt, splits, Hkv): the CTAs that differ only in (query, M tile) walk the same key tiles
 // at the same time, so the pool's K layer is read from DRAM about once and from L2 otherwise.
 template <int D, int PASS>
-__global__ void __launch_bounds__(kRelThreads, 1)
+__global__ void __launch_bounds__(kRelThreads, 2)
 rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const RelParams p) {
   using SM = RelSmem<D>;
   constexpr int SUB = D / 64;
+  constexpr int kStages = kKStages<D>;
   constexpr uint32_t kTileBytes = SM::kTileBytes;
   constexpr uint32_t kIdesc = idesc_bf16_f32(kTile, kTile, 0);
   extern __shared__ unsigned char smem_raw[];
@@ -126,7 +129,7 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (threadIdx.x == 32) {
     mbar_init(bar(kRQFull), 1);
-    for (int i = 0; i < kKStages; ++i) {
+    for (int i = 0; i < kStages; ++i) {
       mbar_init(bar(kRKFull + i), 1);
       mbar_init(bar(kRKEmpty + i), 1);
     }
@@ -144,9 +147,9 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tmem_relinquish();
   }
   if (PASS == 2 && threadIdx.x >= 64) {
-    // rows of the M tile that do not exist get lse = +inf: their 2^(s c - lse) is exactly zero
+    // -lse per query row; rows of the M tile that do not exist get -inf: their 2^(s c - lse) is exactly zero
     const int c = threadIdx.x - 64;
-    lse_s[c] = c < min(kTile, p.rows - mt * kTile) ? p.lse2[(long long)unit * kTile + c] : INFINITY;
+    lse_s[c] = c < min(kTile, p.rows - mt * kTile) ? -p.lse2[(long long)unit * kTile + c] : -INFINITY;
   }
   tc_fence_before();
   __syncthreads();
@@ -164,8 +167,8 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       bool ok = true;
       int i = 0;
       for (; i < n_it && ok; ++i) {
-        const int st = i % kKStages;
-        ok = mbar_wait(bar(kRKEmpty + st), ((i / kKStages) & 1) ^ 1, abort_flag);
+        const int st = i % kStages;
+        ok = mbar_wait(bar(kRKEmpty + st), ((i / kStages) & 1) ^ 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(bar(kRKFull + st), kTileBytes);
 #pragma unroll
@@ -175,8 +178,8 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       if (!ok) {      // gave up: let the copies in flight land before the CTA retires
         mbar_wait(bar(kRQFull), 0, abort_flag + 1);
-        for (int t = max(0, i - kKStages); t < i; ++t)
-          mbar_wait(bar(kRKFull + t % kKStages), (t / kKStages) & 1, abort_flag + 1);
+        for (int t = max(0, i - kStages); t < i; ++t)
+          mbar_wait(bar(kRKFull + t % kStages), (t / kStages) & 1, abort_flag + 1);
       }
     }
     __syncwarp();
@@ -187,8 +190,8 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t q_lo = smem_desc_lo(base + SM::kOffQ, 16);
       bool ok = mbar_wait(bar(kRQFull), 0, abort_flag);
       for (int i = 0; i < n_it && ok; ++i) {
-        const int st = i % kKStages, sb = i & 1;
-        ok = mbar_wait(bar(kRKFull + st), (i / kKStages) & 1, abort_flag) &&
+        const int st = i % kStages, sb = i & 1;
+        ok = mbar_wait(bar(kRKFull + st), (i / kStages) & 1, abort_flag) &&
              mbar_wait(bar(kRSEmpty + sb), ((i >> 1) & 1) ^ 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -243,22 +246,29 @@ rel_pass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           l_run *= rel_ex2(m_run - mx);
           m_run = mx;
         }
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
+        // two scores per FMA / add instruction; the exponentials themselves are one MUFU operation each
+        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), neg_m2 = make_float2(-m_run, -m_run);
+        float2 part[2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll
-        for (int c = 0; c < kTile; ++c) part[c & 3] += rel_ex2(fmaf(s[c], p.scale_log2, -m_run));
-        l_run += (part[0] + part[1]) + (part[2] + part[3]);
+        for (int c = 0; c < kTile; c += 2) {
+          const float2 a = __ffma2_rn(make_float2(s[c], s[c + 1]), scale2, neg_m2);
+          part[(c >> 1) & 1] = __fadd2_rn(part[(c >> 1) & 1], make_float2(rel_ex2(a.x), rel_ex2(a.y)));
+        }
+        l_run += (part[0].x + part[0].y) + (part[1].x + part[1].y);
       } else {
         const long long key = key0 + r;
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
+        const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
+        float2 part[2] = {{0.f, 0.f}, {0.f, 0.f}};
         const float4* lse4 = reinterpret_cast<const float4*>(lse_s);
 #pragma unroll
         for (int c4 = 0; c4 < kTile / 4; ++c4) {
           const float4 l4 = lse4[c4];                     // the same address for every lane: a broadcast
-          const float lv[4] = {l4.x, l4.y, l4.z, l4.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) part[e] += rel_ex2(fmaf(s[4 * c4 + e], p.scale_log2, -lv[e]));
+          const float2 a0 = __ffma2_rn(make_float2(s[4 * c4], s[4 * c4 + 1]), scale2, make_float2(l4.x, l4.y));
+          const float2 a1 = __ffma2_rn(make_float2(s[4 * c4 + 2], s[4 * c4 + 3]), scale2, make_float2(l4.z, l4.w));
+          part[0] = __fadd2_rn(part[0], make_float2(rel_ex2(a0.x), rel_ex2(a0.y)));
+          part[1] = __fadd2_rn(part[1], make_float2(rel_ex2(a1.x), rel_ex2(a1.y)));
         }
-        float v = (part[0] + part[1]) + (part[2] + part[3]);
+        float v = (part[0].x + part[0].y) + (part[1].x + part[1].y);
         int id = -1;
         if (key < p.pool_tokens) id = p.tok_shot[key]; else v = 0.f;
         // shots are runs of consecutive keys: segmented inclusive sum along the lanes, the last
@@ -331,13 +341,24 @@ RelPlan rel_plan(const adapshot_model_t* model, const adapshot_pool_t* pool, int
   pl.n_mt = (pl.rows + kTile - 1) / kTile;
   pl.rows_pad = pl.n_mt * kTile;
   pl.n_tiles = (int)((pool->pool_tokens + kTile - 1) / kTile);
-  // about four resident waves of CTAs, each range at least eight key tiles
+  // Key ranges per unit: units * splits CTAs run in waves of 296 (two per SM on 148 SMs; a fixed
+  // figure, so that the workspace size does not depend on the device), each CTA costs its tiles plus
+  // about four tiles' time of start-up; the split with the cheapest waves * (tiles + 4) is taken,
+  // every range at least eight key tiles.
   const long long units = (long long)B * pl.n_mt * Hkv;
-  long long want = (4ll * 148 + units - 1) / units;
-  const long long most = (pl.n_tiles + 7) / 8;
-  if (want > most) want = most;
-  if (want < 1) want = 1;
-  pl.tiles_per_split = (int)((pl.n_tiles + want - 1) / want);
+  const int most = (pl.n_tiles + 7) / 8 < 256 ? (pl.n_tiles + 7) / 8 : 256;
+  int best_s = 1;
+  long long best_cost = 0;
+  for (int sp = 1; sp <= most; ++sp) {
+    const long long tiles = (pl.n_tiles + sp - 1) / sp;
+    const long long waves = (units * sp + 295) / 296;
+    const long long cost = waves * (tiles + 4);
+    if (sp == 1 || cost < best_cost) {
+      best_s = sp;
+      best_cost = cost;
+    }
+  }
+  pl.tiles_per_split = (pl.n_tiles + best_s - 1) / best_s;
   pl.splits = (pl.n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
   size_t off = 0;
   pl.off_qpack = off;   off += ads_round_up((size_t)B * Hkv * pl.rows_pad * D * 2, 256);
