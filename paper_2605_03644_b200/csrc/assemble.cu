@@ -300,7 +300,8 @@ int launch_gather(GatherArgs a, cudaStream_t st) {
   if (n_sm <= 0) return ADAPSHOT_ECUDA;
   const long long resident_warps = n_sm * 6 * warps_per_block;
   const long long tokens = (long long)a.B * a.ctx_cap;
-  a.run = kRunMax;
+  // a call of one or two layers has little work per token to spread the plan lookup over: longer runs
+  a.run = a.n_layers_call <= 2 ? 4 * kRunMax : kRunMax;
   while (a.run > 1 && tokens / a.run < 4 * resident_warps) a.run >>= 1;
   const long long units = (long long)a.B * ((a.ctx_cap + a.run - 1) / a.run);
   long long blocks = (units + warps_per_block - 1) / warps_per_block;
