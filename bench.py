@@ -113,9 +113,9 @@ NCU_TRAFFIC = {
     # workload: (attn_main bytes per captured launch, layers x queries in that capture,
     #            gather bytes per captured launch, layers x queries in that capture), for the variant
     #            that `--variant auto` picks for the workload
-    "cfg2": (102.0e6, 1, 119.7e6, 1),             # profiles/attn_main_kernel_cfg2.md, profiles/gather_rope_kernel.md
-    "cfg3": (2.2323e9, 16, 2.110e9, 16),          # profiles/attn_main_kernel_cfg3_2layers.md (2 layers x 8 queries, K-only cache)
-    "cfg5": (2.050e9, 4, 1.0684e9, 4),            # profiles/attn_main_and_gather_cfg5_1layer_4queries.md (K-only cache)
+    "cfg2": (102.0e6, 1, 119.6e6, 1),             # profiles/attn_main_kernel_cfg2.md, profiles/gather_rope_kernel.md
+    "cfg3": (2.2323e9, 16, 2.113e9, 16),          # profiles/attn_main_kernel_cfg3_2layers.md (2 layers x 8 queries, K-only cache)
+    "cfg5": (2.049e9, 4, 1.0660e9, 4),            # profiles/attn_main_and_gather_cfg5_1layer_4queries.md (K-only cache)
 }
 
 
