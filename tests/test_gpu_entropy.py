@@ -118,3 +118,44 @@ def test_subset_entropy_reports_a_bad_token_id():
     torch.cuda.synchronize()
     assert st.item() == ab.EINDEX
     assert np.allclose(H.cpu().numpy(), math.log(1000) / 1000, rtol=1e-4)      # the valid token alone
+
+
+@pytest.mark.parametrize("R,V", [(1, 8191), (3, 8192), (3, 8193), (5, 16384), (7, 40001), (300, 24577),
+                                 (1000, 16392), (2, 128256)])
+@pytest.mark.parametrize("dt", [torch.float32, torch.bfloat16])
+def test_entropy_slice_boundaries(R, V, dt):
+    # rows are cut into slices of multiples of 8192 entries: lengths around the unit, a last slice
+    # of a few entries, many rows with several slices each, a few rows with sixteen
+    ab = hp.gpu_binding()
+    g = torch.Generator().manual_seed(R * 131 + V)
+    stride = (V + 7) // 8 * 8
+    scale = torch.linspace(0.5, 5.0, R)[:, None]
+    buf = (torch.randn(R, stride, generator=g) * scale).to(dt)
+    buf[:, V - 1] += 7.0                            # the row maximum sits in the last (shortest) slice
+    H, _, st = hp.run_entropy(ab, buf.cuda()[:, :V], 0.0, 1, want_first=False)
+    want = orc.entropy(hp.f64(buf[:, :V]))
+    assert st == 0
+    assert np.all(np.abs(H.cpu().numpy() - want) <= REL_TOL * np.maximum(want, 1e-3) + 1e-7)
+
+
+@pytest.mark.parametrize("dt", [torch.float32, torch.bfloat16])
+def test_entropy_minus_infinity_conventions(dt):
+    # -inf (and anything at or below -2^97) adds nothing wherever it sits: inside a vector, as a whole
+    # vector, as a whole slice; a row of nothing else has H = 0 by the stated convention
+    ab = hp.gpu_binding()
+    V = 20000
+    x = torch.zeros(5, V)
+    x[0, 3:11] = float("-inf")                      # whole 16-byte vectors and parts of them
+    x[1, :8192] = float("-inf")                     # the whole first slice
+    x[1, 8192:8194] = 1.0                           # two equal survivors beside 11 806 zeros
+    x[2, :] = float("-inf")
+    x[3, :] = -3.0e38
+    x[4, 8192:] = -1.0e30                           # below the floor: counts as -inf
+    got, _, st = hp.run_entropy(ab, x.to(dt).cuda(), 0.0, 1, want_first=False)
+    got = got.cpu().numpy()
+    assert st == 0
+    assert abs(got[0] - math.log(V - 8)) < 1e-4 * math.log(V)
+    want1 = orc.entropy(hp.f64(x[1:2].to(dt)))[0]
+    assert abs(got[1] - want1) < 1e-4 * want1
+    assert got[2] == 0.0 and got[3] == 0.0
+    assert abs(got[4] - math.log(8192)) < 1e-4 * math.log(8192)
