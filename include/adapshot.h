@@ -300,11 +300,10 @@ ADAPSHOT_API int adapshot_decode_attn(const adapshot_model_t* model, const void*
  *   A logit at or below -2^97 (about -1.6e29) counts as -inf: it adds nothing; a row
  *   that holds nothing above it, and an all-NaN row, give H = 0.
  *   Limits: R a multiple of rows_per_group, rows_per_group <= 8192, and
- *   R * splits < 2^31, where splits (one CTA per row and split) is the n in
- *   1..min(64, ceil(V / 4096)) that minimises
- *   ceil(R * n / 1184) * (ceil(V / n) + 1024); ADAPSHOT_ESHAPE otherwise.
+ *   R * splits < 2^31, where splits <= 64 is the number of slices (multiples of 8192
+ *   entries, one CTA each) a row is cut into; ADAPSHOT_ESHAPE otherwise.
  *   Ask adapshot_entropy_workspace_bytes for the scratch size (12 bytes per row and
- *   split, rounded up to 256).                                                   */
+ *   slice, rounded up to 256; it depends on R and V only, not on the device).     */
 ADAPSHOT_API size_t adapshot_entropy_workspace_bytes(int32_t R, int32_t V);
 ADAPSHOT_API int adapshot_entropy(const void* logits, int32_t dtype, int32_t R, int32_t V, int64_t row_stride,
                      float* H, float tau, int32_t rows_per_group, int32_t* first_ok,

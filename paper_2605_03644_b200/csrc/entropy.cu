@@ -118,7 +118,7 @@ entropy_partial_kernel(const T* __restrict__ logits, int V, long long row_stride
   const int r = blockIdx.x / n_split, sp = blockIdx.x % n_split;
   const T* row = logits + (long long)r * row_stride;
   const int begin = sp * slice;
-  const int end = min(V, begin + slice);
+  const int end = V - begin <= slice ? V : begin + slice;      // (begin + slice may not fit an int)
   EntState st{kEntFloor, 0.f, 0.f};    // every logit is at least the floor, so m starts there
 
   const int n_vec = (end - begin) / kVec;                        // slice is a multiple of kVec
@@ -320,17 +320,22 @@ constexpr int kEntCtaOverhead = 2048;    // fixed cost of a CTA (start, state me
 // waves) rather than whole (2.3 waves, the third one a third full), 224 rows as 3 slices (one wave).  `max_states` bounds R * n (the fixed scratch of the static entry point).
 struct EntSplit { int slice, n; };
 EntSplit ent_split(int R, int V, long long max_states = 0x7fffffffll) {
-  const int j_max = (V + kEntSliceUnit - 1) / kEntSliceUnit;     // j_max units: the row in one piece
-  EntSplit best{j_max * kEntSliceUnit, 1};
+  const long long unit = kEntSliceUnit;
+  const long long kMaxSlice = 0x7fffe000ll;                             // the largest multiple of the unit an int holds
+  EntSplit best{(int)((long long)V <= kMaxSlice ? ((long long)V + unit - 1) / unit * unit : kMaxSlice),
+                (long long)V <= kMaxSlice ? 1 : 2};                      // the row in one piece (two beyond 2^31 - 8192)
   double best_cost = 0.0;
-  for (int j = j_max; j >= 1; --j) {
-    const int slice = j * kEntSliceUnit;
-    const int n = (V + slice - 1) / slice;
-    if (n > 64 || (long long)R * n > max_states) break;          // n only grows as j falls
+  for (int want = 1; want <= 64; ++want) {
+    // the shortest slice (a multiple of the unit) that cuts the row into at most `want` pieces
+    const long long per = ((long long)V + want - 1) / want;
+    long long slice = (per + unit - 1) / unit * unit;
+    if (slice > kMaxSlice) slice = kMaxSlice;
+    const int n = (int)(((long long)V + slice - 1) / slice);
+    if ((long long)R * n > max_states) break;                            // n only grows with `want`
     const long long waves = ((long long)R * n + kEntTargetCtas - 1) / kEntTargetCtas;
-    const double cost = (double)waves * (slice + kEntCtaOverhead);
-    if (j == j_max || cost < best_cost) {
-      best = EntSplit{slice, n};
+    const double cost = (double)waves * (double)(slice + kEntCtaOverhead);
+    if (want == 1 || cost < best_cost) {
+      best = EntSplit{(int)slice, n};
       best_cost = cost;
     }
   }
