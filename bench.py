@@ -143,15 +143,20 @@ def resolve_k_by_budget(ab, dpool, q_emb, w: wl.Workload, lengths: np.ndarray) -
     return w.scaled(k=k, probes=(k,))
 
 
-def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 184e9, k_only: bool = False) -> int:
+def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 0.0, k_only: bool = False) -> int:
     """Layers assembled and attended per call: as many as fit beside the pool, the query-side
-    tensors and the outputs, at most 36 GB of assembled K + V (k_only: the cache holds K alone)."""
+    tensors (three times over: device inputs, their end-to-end copies, outputs) and the workspaces,
+    at most 36 GB of assembled K + V (k_only: the cache holds K alone).  device_bytes: the GPU's
+    memory (asked of the current device when 0; 184e9 without one)."""
+    if device_bytes <= 0:
+        device_bytes = (float(torch.cuda.get_device_properties(torch.cuda.current_device()).total_memory)
+                        if torch.cuda.is_available() else 184e9)
     n_tok = float(wl.shot_lengths(w).sum())
     pool_bytes = n_tok * w.bytes_per_token_layer * w.n_layers
     q_bytes = (w.batch * w.n_layers * max(1, len(w.probes)) * w.t_q * (w.n_q_heads + 2 * w.n_kv_heads)
                * w.head_dim * w.elem_size)
     per_layer = float(w.batch) * ctx_cap * w.bytes_per_token_layer * (0.5 if k_only else 1.0)
-    budget = min(36e9, 0.5 * (device_bytes - pool_bytes - 3.0 * q_bytes))
+    budget = min(36e9, 0.6 * (device_bytes - pool_bytes - 3.0 * q_bytes))
     return int(max(1, min(w.n_layers, budget // per_layer)))
 
 
