@@ -117,6 +117,14 @@ def test_maximum_number_of_probe_query_pairs():
     _run_case(w, sel, [1, 2, 4, 6], 1)
 
 
+def test_sixteen_nested_probes():
+    # P = 16 (the most one call takes), every prefix length from one shot to all sixteen, two layers
+    w = wl.CONFIGS["cfg2"].scaled(n_shots=48, len_lo=30, len_hi=200, batch=3, k=16, t_q=24, seed=27)
+    rng = np.random.default_rng(5)
+    sel = np.stack([rng.permutation(48)[:16] for _ in range(3)]).astype(np.int32)
+    _run_case(w, sel, list(range(1, 17)), 2)
+
+
 def test_peaked_scores_rescale_the_accumulator():
     # keys three times larger: scores of a row spread over tens of log2 units, so the row maximum
     # grows by more than the lazy-rescale threshold several times along the context and the
