@@ -157,7 +157,9 @@ def layers_per_call_for(w: wl.Workload, ctx_cap: int, device_bytes: float = 0.0,
                * w.head_dim * w.elem_size)
     per_layer = float(w.batch) * ctx_cap * w.bytes_per_token_layer * (0.5 if k_only else 1.0)
     budget = min(36e9, 0.6 * (device_bytes - pool_bytes - 3.0 * q_bytes))
-    return int(max(1, min(w.n_layers, budget // per_layer)))
+    # at least four chunks where there are layers for it: a caller whose tensors live in host memory
+    # has chunk i + 1 on its way up and chunk i - 1 on its way down while chunk i is computed
+    return int(max(1, min(w.n_layers, budget // per_layer, max(1, -(-w.n_layers // 4)))))
 
 
 def choose_variant(w: wl.Workload, ctx_cap: int, variant: str = "auto", layers_per_call: int = 0):

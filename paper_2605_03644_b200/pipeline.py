@@ -161,11 +161,12 @@ class ReusePath:
 
         host_in / dev_in: {"q_emb", "logits", "q": [...], "kq": [...], "vq": [...]} (one tensor per
         layer chunk), the same shapes on both sides; host_out: {"out": [...], "H", "first_ok",
-        "sel_idx"}.  The query-side tensors go up on a copy stream while selection and the
-        gather run, each chunk's output goes down on another while the next chunk is computed,
-        and the logits go up on the side stream (with entropy_overlap the entropy and its results
-        use it too): PCIe carries both directions at once and the kernels wait only for the bytes
-        they read.  Everything is
+        "sel_idx"}.  Every upload goes through one copy stream in the order it is needed (query
+        embeddings, the chunks' query-side tensors, the logits), every download through another
+        (the selection, each chunk's output while the next chunk is computed, the entropies); the
+        compute stream issues no copy itself and waits only for the bytes its next kernel reads
+        (with entropy_overlap the logits, the entropy step and its results use the side stream).
+        PCIe carries both directions at once.  Everything is
         joined back to the current stream before returning (the results are complete once that
         stream is synchronised), so the pass can also be captured into a graph."""
         if self.overlap:
@@ -176,26 +177,41 @@ class ReusePath:
             self.ev_in = [torch.cuda.Event() for _ in self.chunks]
             self.ev_out = [torch.cuda.Event() for _ in self.chunks]
             self.ev_d2h = torch.cuda.Event()
+            self.ev_qemb, self.ev_sel = torch.cuda.Event(), torch.cuda.Event()
         main = torch.cuda.current_stream()
         self.ev_begin.record(main)
-        for s in (self.side, self.h2d, self.d2h):
+        for s in (self.h2d, self.d2h) + ((self.side,) if self.entropy_overlap else ()):
             s.wait_event(self.ev_begin)
-        with torch.cuda.stream(self.side):
-            dev_in["logits"].copy_(host_in["logits"], non_blocking=True)
-            if self.entropy_overlap:
+        # The compute stream issues no copy of its own: a copy waits in its engine's queue behind
+        # whatever was submitted to that engine before, and a few KB stuck behind gigabytes would stall
+        # the kernels that follow it in the stream.  Uploads go through the h2d stream in the order
+        # they are needed (the query embeddings first, the logits last unless the entropy step runs
+        # beside the pass), downloads through the d2h stream.
+        with torch.cuda.stream(self.h2d):
+            dev_in["q_emb"].copy_(host_in["q_emb"], non_blocking=True)
+            self.ev_qemb.record(self.h2d)
+        if self.entropy_overlap:
+            with torch.cuda.stream(self.side):
+                dev_in["logits"].copy_(host_in["logits"], non_blocking=True)
                 self.entropy(dev_in["logits"], tau)
                 host_out["H"].copy_(self.H, non_blocking=True)
                 host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
-            self.ev_entropy.record(self.side)
+                self.ev_entropy.record(self.side)
         with torch.cuda.stream(self.h2d):
             for i in range(len(self.chunks)):
                 for name in ("q", "kq", "vq"):
                     dev_in[name][i].copy_(host_in[name][i], non_blocking=True)
                 self.ev_in[i].record(self.h2d)
-        dev_in["q_emb"].copy_(host_in["q_emb"], non_blocking=True)
+            if not self.entropy_overlap:      # needed only after the last attention call: behind the bulk
+                dev_in["logits"].copy_(host_in["logits"], non_blocking=True)
+                self.ev_entropy.record(self.h2d)
+        main.wait_event(self.ev_qemb)
         self.select(dev_in["q_emb"])
         self.plan()
-        host_out["sel_idx"].copy_(self.sel_idx, non_blocking=True)
+        self.ev_sel.record(main)
+        with torch.cuda.stream(self.d2h):
+            self.d2h.wait_event(self.ev_sel)
+            host_out["sel_idx"].copy_(self.sel_idx, non_blocking=True)
         for i, (lb, le) in enumerate(self.chunks):
             if not self.fused:
                 self.assemble(lb, le, keep_plan=True)
@@ -211,8 +227,11 @@ class ReusePath:
         main.wait_event(self.ev_entropy)
         if not self.entropy_overlap:          # the logits are up; the probe follows the last attention call
             self.entropy(dev_in["logits"], tau)
-            host_out["H"].copy_(self.H, non_blocking=True)
-            host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
+            self.ev_sel.record(main)
+            with torch.cuda.stream(self.d2h):
+                self.d2h.wait_event(self.ev_sel)
+                host_out["H"].copy_(self.H, non_blocking=True)
+                host_out["first_ok"].copy_(self.first_ok, non_blocking=True)
         self.ev_d2h.record(self.d2h)
         main.wait_event(self.ev_d2h)
         return host_out
