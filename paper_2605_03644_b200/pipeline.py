@@ -20,11 +20,29 @@ import torch
 from . import binding as ab
 
 
+def layer_chunks(n_layers: int, lpc: int, ramp: bool = False):
+    """Layer ranges of one pass: chunks of lpc layers; with ramp (and room for it) the first and the last
+    chunk are a quarter of that and their neighbours make up for it ([s, lpc - s, lpc, ..., lpc - s, s]).
+    For a caller whose tensors live in host memory the first chunk's upload and the last chunk's download
+    are the only copies no kernel runs beside, so they are kept short."""
+    small = max(1, lpc // 4)
+    if not ramp or lpc < 2 or n_layers < 2 * lpc:
+        sizes = [min(lpc, n_layers - lb) for lb in range(0, n_layers, lpc)]
+    else:
+        middle = n_layers - 2 * lpc
+        sizes = [small, lpc - small] + [min(lpc, middle - lb) for lb in range(0, middle, lpc)] + [lpc - small, small]
+    out, lb = [], 0
+    for n in sizes:
+        out.append((lb, lb + n))
+        lb += n
+    return out
+
+
 class ReusePath:
     def __init__(self, model: ab.ModelT, pool: ab.Pool, batch: int, k: int, probes: Sequence[int],
                  t_q: int, vocab: int, ctx_cap: int, layers_per_call: Optional[int] = None,
                  overlap: bool = False, fused: bool = False, entropy_overlap: bool = False,
-                 vpool: Optional[bool] = False, device="cuda"):
+                 vpool: Optional[bool] = False, ramp: bool = False, device="cuda"):
         self.model, self.pool = model, pool
         self.B, self.k, self.probes, self.t_q, self.vocab = batch, k, list(probes), t_q, vocab
         self.P = len(self.probes)
@@ -38,7 +56,7 @@ class ReusePath:
         self.sel_idx = torch.empty((batch, k), dtype=torch.int32, device=device)
         self.sel_score = torch.empty((batch, k), dtype=torch.float32, device=device)
         self.ctx_off = torch.empty((batch, k + 1), dtype=torch.int64, device=device)
-        self.chunks = [(lb, min(self.nl, lb + self.lpc)) for lb in range(0, self.nl, self.lpc)]
+        self.chunks = layer_chunks(self.nl, self.lpc, ramp)
         self.fused = bool(fused)
         if vpool is None:
             # measured choice: a cache that stays in L2 between the gather and the attention (a single

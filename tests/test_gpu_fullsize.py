@@ -94,8 +94,8 @@ def _fullsize(name, n_combos=6, rows_per_combo=44, n_blocks=64, seed=0, fused=Fa
         b, l, g = int(rng.integers(w.batch)), int(rng.integers(w.n_layers)), int(rng.integers(w.n_kv_heads))
         L_max = int(off[b, w.probes[-1]])
         k_ctx, v_ctx = _context_of(pool, sel[b], l, g, L_max, w.rope_base)
-        ci = l // lpc
-        out_l = path.out[ci][b, l - ci * lpc]
+        ci = next(i for i, (lb, le) in enumerate(path.chunks) if lb <= l < le)
+        out_l = path.out[ci][b, l - path.chunks[ci][0]]
         kq, vq = hp.f64(qs["kq"][b, l][:, :, g:g + 1]), hp.f64(qs["vq"][b, l][:, :, g:g + 1])
         for _ in range(rows_per_combo):
             j, t, hh = int(rng.integers(len(w.probes))), int(rng.integers(w.t_q)), int(rng.integers(G))

@@ -32,3 +32,18 @@ def test_small_pool_and_queries_are_reproducible():
     assert p2["k"].dtype == torch.bfloat16 and p2["pool_tokens"] == int(p2["shot_off"][-1])
     x = wl.to_f64(p2["k"])
     assert x.dtype == np.float64 and np.array_equal(x.astype(np.float32), p2["k"].float().numpy())
+
+
+def test_layer_chunks_cover_the_layers_in_order():
+    from paper_2605_03644_b200.pipeline import layer_chunks
+    for n in (1, 2, 3, 7, 8, 32, 80):
+        for lpc in (1, 2, 3, 4, 8, 20, 32, 80):
+            for ramp in (False, True):
+                c = layer_chunks(n, lpc, ramp)
+                assert c[0][0] == 0 and c[-1][1] == n
+                assert all(a[1] == b[0] for a, b in zip(c, c[1:]))
+                assert all(0 < e - b <= lpc for b, e in c)
+    assert [e - b for b, e in layer_chunks(32, 4, True)] == [1, 3, 4, 4, 4, 4, 4, 4, 3, 1]
+    assert [e - b for b, e in layer_chunks(32, 8, True)] == [2, 6, 8, 8, 6, 2]
+    assert [e - b for b, e in layer_chunks(32, 32, True)] == [32]
+    assert [e - b for b, e in layer_chunks(32, 8, False)] == [8, 8, 8, 8]
