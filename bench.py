@@ -616,6 +616,33 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
     e2e_ms, _ = job_aggregate(e2e_ms, 0.0, dist, dev)
     e2e_value = job_tokens / (e2e_ms / n_e2e * 1e-3)
     check_status("after the end-to-end pass")
+    e2e_timeline = None
+    if args.e2e_timeline:
+        # when each step of one plain (uncaptured) end-to-end pass ends on the compute stream, from events
+        # recorded after the calls; the copies run on their own streams beside them
+        marks = []
+        def wrapped(name, fn):
+            def call(*a, **k):
+                r = fn(*a, **k)
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                marks.append((name, e))
+                return r
+            return call
+        names = ["select", "plan", "assemble", "attend", "attend_fused", "entropy"]
+        saved = {n: getattr(path, n) for n in names}
+        for n in names:
+            setattr(path, n, wrapped(n, saved[n]))
+        flush.zero_()
+        t0 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        path.run_host(host, dev_in, host_out, args.tau)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t1.record()
+        torch.cuda.synchronize()
+        for n in names:
+            setattr(path, n, saved[n])
+        e2e_timeline = [[n, t0.elapsed_time(e)] for n, e in marks] + [["results in host memory", t0.elapsed_time(t1)]]
 
     config = workload_config(w, pool["n_shots"], pool["pool_tokens"], counts["ctx_tokens"], world)
     config.update({"variant": "fused" if fused else ("vpool" if vpool else "materialise"), "k_pos_mode": args.k_pos_mode, "cuda_graph": use_graph,
@@ -635,6 +662,7 @@ def measure(args, name: str, steps: int, warmup: int, dev, peaks, dist, rank: in
         "per_call_ms": per_call_ms,
         "step_ms_min_med_max": [float(step_ms.min()), float(np.median(step_ms)), float(step_ms.max())],
         "timed_region_ms": total_ms,
+        **({"e2e_timeline_ms": e2e_timeline} if e2e_timeline is not None else {}),
     }
     if per_probe is not None:
         res["per_probe"] = per_probe
@@ -807,6 +835,8 @@ def main():
                     help="replay the pass as one CUDA graph (auto: single-layer workloads)")
     ap.add_argument("--entropy-overlap", action="store_true",
                     help="run the entropy probe on a side stream beside the pass instead of after the attention")
+    ap.add_argument("--e2e-timeline", action="store_true",
+                    help="add e2e_timeline_ms to the line: when every step of one end-to-end pass ends")
     ap.add_argument("--ramp", action="store_true",
                     help="make the first and the last layer chunk of a pass a quarter of --layers-per-call: it shortens "
                          "the only upload and download of the end-to-end pass that no kernel runs beside (measured: "
